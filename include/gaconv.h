@@ -1,0 +1,153 @@
+/*
+ * gaconv -- filter-gradient (dW) convolution of a conv layer's backward pass on one NVIDIA B200
+ * (sm_100a), exact and in the approximated forms of "Accelerated CNN Training Through Gradient
+ * Approximation" (arXiv 1908.05460), Section 2.
+ *
+ * Notation.  X[n,c,h,w] input activations (paper: I), dY[n,k,p,q] output gradient (paper: dO),
+ * dW[k,c,r,s] filter gradient (paper: df); paper symbols K = r = s, C_i = c, C_o = k (Section 2.4).
+ *   P = (H + 2*pad_h - R)/stride_h + 1,  Q = (W + 2*pad_w - S)/stride_w + 1.
+ *
+ * Conventions of every entry point
+ *   - Plain C ABI: status codes only, nothing throws, nothing aborts.
+ *   - Every pointer named x, dy, dw, idx, sum, dy_sparse, workspace or *_dev is DEVICE memory on the
+ *     current CUDA device, allocated and freed by the caller, 16-byte aligned.  Pointers named *_host
+ *     are host memory (pinned for true asynchrony).  The library allocates no device memory and keeps
+ *     no reference to any buffer after the call returns (the work itself is asynchronous, see below).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it; no entry point
+ *     synchronises the host except gaconv_poll_async_status and gaconv_dw_from_host's final wait.
+ *   - Validation errors are returned at once and enqueue nothing.
+ *   - dw is overwritten (no accumulate-into).  It is always fp32.
+ *   - Same inputs, descriptor and seed give bitwise identical outputs from run to run: every
+ *     reduction has a fixed order.
+ */
+#ifndef GACONV_H
+#define GACONV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GACONV_OK = 0,
+    GACONV_ERR_NULL_POINTER = 1,
+    GACONV_ERR_BAD_DESC = 2,          /* non-positive size, P or Q < 1, unknown enum, wrong struct_size */
+    GACONV_ERR_UNSUPPORTED = 3,       /* valid request this build has no kernel for                      */
+    GACONV_ERR_MISALIGNED = 4,        /* a device pointer is not 16-byte aligned                          */
+    GACONV_ERR_WORKSPACE_TOO_SMALL = 5,
+    GACONV_ERR_CUDA = 6,              /* a CUDA runtime call failed; see cudaGetLastError                 */
+    GACONV_ERR_TIMEOUT = 7            /* a bounded device-side wait gave up (read by the poll call)       */
+} gaconv_status_t;
+
+typedef enum { GACONV_F32 = 0, GACONV_BF16 = 1 } gaconv_dtype_t;            /* of x and dy            */
+typedef enum { GACONV_X_NHWC = 0, GACONV_X_NCHW = 1 } gaconv_x_layout_t;    /* NHWC: Section 2.4     */
+typedef enum { GACONV_DY_NKPQ = 0 } gaconv_dy_layout_t;                     /* = N C_o H W           */
+typedef enum { GACONV_DW_KRSC = 0, GACONV_DW_KCRS = 1 } gaconv_dw_layout_t; /* KRSC = C_o K K C_i    */
+typedef enum { GACONV_METHOD_EXACT = -1, GACONV_METHOD_ZERO = 0, GACONV_METHOD_RANDOM = 1,
+               GACONV_METHOD_TOP1 = 2 } gaconv_method_t;
+/* arithmetic of the exact contraction */
+typedef enum {
+    GACONV_MATH_DEFAULT = 0,   /* bf16 inputs: bf16 tensor cores, fp32 accumulate; fp32 inputs: fp32-accurate */
+    GACONV_MATH_TF32 = 1       /* fp32 inputs only: one TF32 tensor-core pass (operands cut to 10 mantissa bits) */
+} gaconv_math_t;
+/* kernel family; AUTO picks the fastest that supports the shape */
+typedef enum { GACONV_ALGO_AUTO = 0, GACONV_ALGO_DIRECT = 1, GACONV_ALGO_TENSOR = 2 } gaconv_algo_t;
+
+/* Problem statement of one layer (Section 2.4: "input tensor I and output gradient tensor dO"). */
+typedef struct gaconv_conv_desc {
+    uint32_t struct_size;              /* = sizeof(gaconv_conv_desc_t); versions the struct               */
+    int32_t  n, c, h, w;               /* X is n x c x h x w                                              */
+    int32_t  k, r, s;                  /* k filters of r x s (dilation 1, one group)                      */
+    int32_t  stride_h, stride_w, pad_h, pad_w;
+    int32_t  in_dtype;                 /* gaconv_dtype_t of x and dy                                      */
+    int32_t  x_layout, dy_layout, dw_layout;
+    int32_t  math;                     /* gaconv_math_t                                                   */
+    int32_t  algo;                     /* gaconv_algo_t                                                   */
+    float    alpha;                    /* dw = alpha * (...); 1 for parity, 1/128 in the paper's runs (Section 2.3) */
+    float    rand_std;                 /* METHOD_RANDOM: standard deviation; the paper uses 1/128 (Section 2.2)     */
+    void    *workspace;                /* device scratch prepared by gaconv_workspace_init                */
+    size_t   workspace_bytes;
+} gaconv_conv_desc_t;
+
+const char *gaconv_status_string(gaconv_status_t status);
+
+/* Device scratch one call needs for `method` (GACONV_METHOD_EXACT for the exact path) with this
+ * descriptor (its workspace fields are ignored).  Never fails for a valid descriptor; *bytes > 0. */
+gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t *desc, int32_t method, size_t *bytes);
+
+/* Prepare a workspace once after allocating it (zero-fills its control words).  Afterwards the
+ * workspace may be reused by any number of calls that do not overlap on the GPU; each call leaves the
+ * control words as it found them.  Two calls running concurrently must use two workspaces. */
+gaconv_status_t gaconv_workspace_init(void *workspace, size_t bytes, void *stream);
+
+/* Exact filter gradient (the operation marked in the paper's Figure 1; Section 2.4):
+ *   dw[k,c,r,s] = alpha * sum_{n,p,q} Xz[n,c,p*stride_h+r-pad_h,q*stride_w+s-pad_w] * dy[n,k,p,q]
+ * with Xz = x, zero outside the image; cross-correlation, no filter flip.
+ * x: n*c*h*w elements of in_dtype in x_layout; dy: n*k*p*q elements in dy_layout; dw: k*c*r*s floats
+ * in dw_layout (written).  Errors: NULL_POINTER, BAD_DESC, MISALIGNED, UNSUPPORTED,
+ * WORKSPACE_TOO_SMALL, CUDA. */
+gaconv_status_t gaconv_dw_exact(const void *x, const void *dy, float *dw,
+                                const gaconv_conv_desc_t *desc, void *stream);
+
+/* Approximated filter gradient, Section 2:
+ *   GACONV_METHOD_ZERO   (2.1)  dw = +0.
+ *   GACONV_METHOD_RANDOM (2.2)  dw[i] = rand_std * z_i, z_i independent standard normals drawn from
+ *        Philox-4x32-10 keyed by `seed` (counter j gives elements 4j..4j+3 by Box-Muller; i runs over
+ *        the logical [k][c][r][s] order whatever dw_layout is).  Pass a new seed per layer and batch:
+ *        the paper regenerates the values every batch.  x and dy may be NULL.
+ *   GACONV_METHOD_TOP1   (2.3, Algorithm 1)  for every (n,k): keep only the largest-magnitude entry of
+ *        dy[n,k,:,:] (lowest p*Q+q among equals), replace it by the signed sum of the map, and take
+ *        the exact filter gradient of that sparse tensor.
+ * `seed` is ignored by ZERO and TOP1. */
+gaconv_status_t gaconv_dw_approx(int32_t method, const void *x, const void *dy, float *dw,
+                                 const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
+
+/* Selection step of Algorithm 1 alone ("arg max abs" and "sum" lines), for inspection:
+ *   idx[n*K+k] = p*Q+q of the retained entry, sum[n*K+k] = signed sum of dy[n,k,:,:] (fp32).
+ * dy_sparse (may be NULL) receives the dense sparse tensor in dy's dtype and layout: the sum, rounded
+ * to in_dtype, at the retained position and zero elsewhere.  Needs no workspace. */
+gaconv_status_t gaconv_approx_select(const void *dy, int32_t *idx, float *sum, void *dy_sparse,
+                                     const gaconv_conv_desc_t *desc, void *stream);
+
+/* Same operation as gaconv_dw_exact / gaconv_dw_approx (method as above, GACONV_METHOD_EXACT for
+ * exact) with HOST inputs and output: copies x_host and dy_host into the caller's device staging
+ * buffers x_dev and dy_dev, runs, copies dw_dev back into dw_host, and waits for the stream.  The
+ * host-to-device and device-to-host transfers are part of the call.  The paper's operator has the
+ * same shape: activations and gradients in, filter gradient out (Section 2.4). */
+gaconv_status_t gaconv_dw_from_host(int32_t method, const void *x_host, const void *dy_host, float *dw_host,
+                                    void *x_dev, void *dy_dev, float *dw_dev,
+                                    const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
+
+/* Waits for `stream`, then reports GACONV_ERR_TIMEOUT if a kernel that used desc->workspace gave up
+ * on a bounded wait since the last poll (and clears the flag), GACONV_OK otherwise. */
+gaconv_status_t gaconv_poll_async_status(const gaconv_conv_desc_t *desc, void *stream);
+
+/* ---- approximation schedules (Section 2.5): which method each layer uses at each training batch ---- */
+typedef struct gaconv_schedule gaconv_schedule_t;   /* host object, owned by the caller via create/destroy */
+typedef enum {
+    GACONV_SCHED_EVERY_4TH_LAYER = 0,            /* Section 3: every 4th conv from the 2nd, every batch      */
+    GACONV_SCHED_ALT_LAYER_ALT_BATCH = 1,        /* Section 3.4 schedule 2: even layers on odd steps         */
+    GACONV_SCHED_ALL_LAYERS_EVERY_4TH_BATCH = 2, /* Section 3.4 schedule 3: all layers when step % 4 == 3    */
+    GACONV_SCHED_LAYER2_ALT_BATCH = 3,           /* Section 3, two-layer CNN: conv 2 on odd steps            */
+    GACONV_SCHED_SEEDED_FRACTION_ALT_BATCH = 4   /* round(fraction*L) layers with the lowest
+                                                    splitmix64(seed+layer), approximated on odd steps       */
+} gaconv_sched_kind_t;
+
+gaconv_status_t gaconv_schedule_create(gaconv_schedule_t **out, int32_t num_layers, int32_t kind,
+                                       int32_t method, double fraction, uint64_t seed);
+/* Method of `layer` (0-based) at training step `step` (0-based): GACONV_METHOD_EXACT or the
+ * schedule's approximation method; -2 on bad arguments. */
+int32_t gaconv_schedule_method(const gaconv_schedule_t *sched, int32_t layer, int64_t step);
+/* Decide and dispatch one layer of one step: gaconv_dw_exact or gaconv_dw_approx(method) on `stream`;
+ * the random method is seeded with a mix of (schedule seed, step, layer) so values change every batch. */
+gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t *sched, int32_t layer, int64_t step,
+                                          const void *x, const void *dy, float *dw,
+                                          const gaconv_conv_desc_t *desc, void *stream);
+void gaconv_schedule_destroy(gaconv_schedule_t *sched);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GACONV_H */

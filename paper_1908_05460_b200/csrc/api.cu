@@ -1,0 +1,301 @@
+// C-ABI entry points of libgaconv: argument validation, workspace planning, kernel dispatch and the
+// approximation-schedule driver (paper Section 2.5).  Every step of the path runs in this library's
+// kernels; there is no CPU or library fallback.
+#include <new>
+
+#include "gaconv_internal.h"
+
+using namespace gaconv;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
+{
+    if (d == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (d->struct_size != sizeof(gaconv_conv_desc_t)) return GACONV_ERR_BAD_DESC;
+    if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1 || d->k < 1 || d->r < 1 || d->s < 1) return GACONV_ERR_BAD_DESC;
+    if (d->stride_h < 1 || d->stride_w < 1 || d->pad_h < 0 || d->pad_w < 0) return GACONV_ERR_BAD_DESC;
+    if (d->h + 2 * d->pad_h < d->r || d->w + 2 * d->pad_w < d->s) return GACONV_ERR_BAD_DESC;
+    if (d->in_dtype != GACONV_F32 && d->in_dtype != GACONV_BF16) return GACONV_ERR_BAD_DESC;
+    if (d->x_layout != GACONV_X_NHWC && d->x_layout != GACONV_X_NCHW) return GACONV_ERR_BAD_DESC;
+    if (d->dy_layout != GACONV_DY_NKPQ) return GACONV_ERR_BAD_DESC;
+    if (d->dw_layout != GACONV_DW_KRSC && d->dw_layout != GACONV_DW_KCRS) return GACONV_ERR_BAD_DESC;
+    if (d->math != GACONV_MATH_DEFAULT && d->math != GACONV_MATH_TF32) return GACONV_ERR_BAD_DESC;
+    if (d->algo < GACONV_ALGO_AUTO || d->algo > GACONV_ALGO_TENSOR) return GACONV_ERR_BAD_DESC;
+    g->n = d->n; g->c = d->c; g->h = d->h; g->w = d->w; g->k = d->k; g->r = d->r; g->s = d->s;
+    g->stride_h = d->stride_h; g->stride_w = d->stride_w; g->pad_h = d->pad_h; g->pad_w = d->pad_w;
+    g->p = (d->h + 2 * d->pad_h - d->r) / d->stride_h + 1;
+    g->q = (d->w + 2 * d->pad_w - d->s) / d->stride_w + 1;
+    if (g->p < 1 || g->q < 1) return GACONV_ERR_BAD_DESC;
+    // element counts must fit comfortably in 63 bits and per-map sizes in 31
+    if ((long long)g->p * g->q > (1ll << 30) || (long long)g->r * g->s * g->c > (1ll << 30)) return GACONV_ERR_UNSUPPORTED;
+    if (d->x_layout == GACONV_X_NHWC) {
+        g->xs_c = 1; g->xs_w = d->c; g->xs_h = (long long)d->w * d->c; g->xs_n = (long long)d->h * d->w * d->c;
+    } else {
+        g->xs_w = 1; g->xs_h = d->w; g->xs_c = (long long)d->h * d->w; g->xs_n = (long long)d->c * d->h * d->w;
+    }
+    if (d->dw_layout == GACONV_DW_KRSC) {
+        g->ws_c = 1; g->ws_s = d->c; g->ws_r = (long long)d->s * d->c; g->ws_k = (long long)d->r * d->s * d->c;
+    } else {
+        g->ws_s = 1; g->ws_r = d->s; g->ws_c = (long long)d->r * d->s; g->ws_k = (long long)d->c * d->r * d->s;
+    }
+    g->bf16 = d->in_dtype == GACONV_BF16;
+    g->alpha = d->alpha;
+    return GACONV_OK;
+}
+
+struct Top1Layout { size_t idx_off, sum_off, partial_off, total; GatherPlan gp; };
+Top1Layout top1_layout(const Geom& g)
+{
+    Top1Layout L;
+    L.gp = plan_gather(g);
+    const size_t maps = (size_t)g.n * g.k;
+    L.idx_off = kWsDataOffset;
+    L.sum_off = align_up(L.idx_off + maps * sizeof(int32_t), 256);
+    L.partial_off = align_up(L.sum_off + maps * sizeof(float), 256);
+    L.total = align_up(L.partial_off + L.gp.partial_bytes, 256);
+    return L;
+}
+
+struct ExactLayout { size_t partial_off, total; DirectPlan dp; };
+ExactLayout exact_layout(const Geom& g)
+{
+    ExactLayout L;
+    L.dp = plan_direct(g);
+    L.partial_off = kWsDataOffset;
+    L.total = align_up(L.partial_off + L.dp.partial_bytes, 256);
+    return L;
+}
+
+gaconv_status_t check_ws(const gaconv_conv_desc_t* d, size_t need)
+{
+    if (d->workspace == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(d->workspace)) return GACONV_ERR_MISALIGNED;
+    if (d->workspace_bytes < need) return GACONV_ERR_WORKSPACE_TOO_SMALL;
+    return GACONV_OK;
+}
+
+uint64_t splitmix64(uint64_t x)
+{
+    uint64_t z = x + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+}  // namespace
+
+struct gaconv_schedule {
+    int32_t num_layers, kind, method;
+    double fraction;
+    uint64_t seed;
+    bool* mask;   // SEEDED_FRACTION: layers in the approximated subset
+};
+
+extern "C" {
+
+const char* gaconv_status_string(gaconv_status_t s)
+{
+    switch (s) {
+        case GACONV_OK: return "ok";
+        case GACONV_ERR_NULL_POINTER: return "null pointer";
+        case GACONV_ERR_BAD_DESC: return "bad descriptor";
+        case GACONV_ERR_UNSUPPORTED: return "unsupported request";
+        case GACONV_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+        case GACONV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case GACONV_ERR_CUDA: return "CUDA error";
+        case GACONV_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t method, size_t* bytes)
+{
+    if (bytes == nullptr) return GACONV_ERR_NULL_POINTER;
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    switch (method) {
+        case GACONV_METHOD_EXACT: *bytes = exact_layout(g).total; return GACONV_OK;
+        case GACONV_METHOD_TOP1: *bytes = top1_layout(g).total; return GACONV_OK;
+        case GACONV_METHOD_ZERO:
+        case GACONV_METHOD_RANDOM: *bytes = kWsDataOffset; return GACONV_OK;
+    }
+    return GACONV_ERR_BAD_DESC;
+}
+
+gaconv_status_t gaconv_workspace_init(void* workspace, size_t bytes, void* stream)
+{
+    if (workspace == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(workspace)) return GACONV_ERR_MISALIGNED;
+    if (bytes < kWsDataOffset) return GACONV_ERR_WORKSPACE_TOO_SMALL;
+    if (cudaMemsetAsync(workspace, 0, kWsDataOffset, static_cast<cudaStream_t>(stream)) != cudaSuccess) return GACONV_ERR_CUDA;
+    return GACONV_OK;
+}
+
+gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const gaconv_conv_desc_t* desc, void* stream)
+{
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
+    if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
+    if (desc->algo == GACONV_ALGO_TENSOR || desc->math == GACONV_MATH_TF32) return GACONV_ERR_UNSUPPORTED;
+    const ExactLayout L = exact_layout(g);
+    st = check_ws(desc, L.total);
+    if (st != GACONV_OK) return st;
+    char* ws = static_cast<char*>(desc->workspace);
+    cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
+                                  reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.dp,
+                                  static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+}
+
+gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, float* dw,
+                                 const gaconv_conv_desc_t* desc, uint64_t seed, void* stream)
+{
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    if (dw == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(dw)) return GACONV_ERR_MISALIGNED;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t count = (size_t)g.k * g.c * g.r * g.s;
+    if (method == GACONV_METHOD_ZERO) return launch_zero(dw, count, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    if (method == GACONV_METHOD_RANDOM)
+        return launch_random(dw, g, seed, desc->rand_std, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    if (method != GACONV_METHOD_TOP1) return GACONV_ERR_BAD_DESC;
+    if (x == nullptr || dy == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(x) || !aligned16(dy)) return GACONV_ERR_MISALIGNED;
+    const Top1Layout L = top1_layout(g);
+    st = check_ws(desc, L.total);
+    if (st != GACONV_OK) return st;
+    char* ws = static_cast<char*>(desc->workspace);
+    int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx_off);
+    float* sum = reinterpret_cast<float*>(ws + L.sum_off);
+    if (launch_select(dy, idx, sum, nullptr, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (launch_gather(x, idx, sum, dw, reinterpret_cast<float*>(ws + L.partial_off),
+                      reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, cs) != cudaSuccess)
+        return GACONV_ERR_CUDA;
+    return GACONV_OK;
+}
+
+gaconv_status_t gaconv_approx_select(const void* dy, int32_t* idx, float* sum, void* dy_sparse,
+                                     const gaconv_conv_desc_t* desc, void* stream)
+{
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    if (dy == nullptr || idx == nullptr || sum == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(dy) || !aligned16(idx) || !aligned16(sum) || !aligned16(dy_sparse)) return GACONV_ERR_MISALIGNED;
+    return launch_select(dy, idx, sum, dy_sparse, g, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GACONV_OK
+                                                                                                         : GACONV_ERR_CUDA;
+}
+
+gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
+                                    void* x_dev, void* dy_dev, float* dw_dev, const gaconv_conv_desc_t* desc,
+                                    uint64_t seed, void* stream)
+{
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    if (dw_host == nullptr || dw_dev == nullptr) return GACONV_ERR_NULL_POINTER;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const bool needs_inputs = method == GACONV_METHOD_EXACT || method == GACONV_METHOD_TOP1;
+    if (needs_inputs) {
+        if (x_host == nullptr || dy_host == nullptr || x_dev == nullptr || dy_dev == nullptr) return GACONV_ERR_NULL_POINTER;
+        const size_t eb = g.bf16 ? 2 : 4;
+        if (cudaMemcpyAsync(x_dev, x_host, (size_t)g.n * g.c * g.h * g.w * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+            cudaMemcpyAsync(dy_dev, dy_host, (size_t)g.n * g.k * g.p * g.q * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+            return GACONV_ERR_CUDA;
+    }
+    st = method == GACONV_METHOD_EXACT ? gaconv_dw_exact(x_dev, dy_dev, dw_dev, desc, stream)
+                                       : gaconv_dw_approx(method, x_dev, dy_dev, dw_dev, desc, seed, stream);
+    if (st != GACONV_OK) return st;
+    if (cudaMemcpyAsync(dw_host, dw_dev, (size_t)g.k * g.c * g.r * g.s * sizeof(float), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+        return GACONV_ERR_CUDA;
+    return cudaStreamSynchronize(cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+}
+
+gaconv_status_t gaconv_poll_async_status(const gaconv_conv_desc_t* desc, void* stream)
+{
+    if (desc == nullptr || desc->workspace == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (desc->workspace_bytes < kWsDataOffset) return GACONV_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, desc->workspace, sizeof(word), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (word == 0) return GACONV_OK;
+    if (cudaMemsetAsync(desc->workspace, 0, sizeof(word), cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    return GACONV_ERR_TIMEOUT;
+}
+
+// ---- approximation schedules ----------------------------------------------------------------
+
+gaconv_status_t gaconv_schedule_create(gaconv_schedule_t** out, int32_t num_layers, int32_t kind, int32_t method,
+                                       double fraction, uint64_t seed)
+{
+    if (out == nullptr) return GACONV_ERR_NULL_POINTER;
+    *out = nullptr;
+    if (num_layers < 1 || num_layers > (1 << 20)) return GACONV_ERR_BAD_DESC;
+    if (kind < GACONV_SCHED_EVERY_4TH_LAYER || kind > GACONV_SCHED_SEEDED_FRACTION_ALT_BATCH) return GACONV_ERR_BAD_DESC;
+    if (method != GACONV_METHOD_ZERO && method != GACONV_METHOD_RANDOM && method != GACONV_METHOD_TOP1) return GACONV_ERR_BAD_DESC;
+    if (!(fraction >= 0.0 && fraction <= 1.0)) return GACONV_ERR_BAD_DESC;
+    gaconv_schedule* s = new (std::nothrow) gaconv_schedule{num_layers, kind, method, fraction, seed, nullptr};
+    if (s == nullptr) return GACONV_ERR_BAD_DESC;
+    if (kind == GACONV_SCHED_SEEDED_FRACTION_ALT_BATCH) {
+        s->mask = new (std::nothrow) bool[num_layers]();
+        uint64_t* hash = new (std::nothrow) uint64_t[num_layers];
+        if (s->mask == nullptr || hash == nullptr) { delete[] s->mask; delete[] hash; delete s; return GACONV_ERR_BAD_DESC; }
+        for (int l = 0; l < num_layers; ++l) hash[l] = splitmix64(seed + (uint64_t)l);
+        int m = (int)(fraction * num_layers + 0.5);
+        if (m > num_layers) m = num_layers;
+        // a layer is chosen when fewer than m layers precede it in (hash, index) order
+        for (int l = 0; l < num_layers; ++l) {
+            int before = 0;
+            for (int o = 0; o < num_layers; ++o)
+                if (hash[o] < hash[l] || (hash[o] == hash[l] && o < l)) ++before;
+            s->mask[l] = before < m;
+        }
+        delete[] hash;
+    }
+    *out = s;
+    return GACONV_OK;
+}
+
+int32_t gaconv_schedule_method(const gaconv_schedule_t* s, int32_t layer, int64_t step)
+{
+    if (s == nullptr || layer < 0 || layer >= s->num_layers || step < 0) return -2;
+    const int one_based = layer + 1;
+    bool approx = false;
+    switch (s->kind) {
+        case GACONV_SCHED_EVERY_4TH_LAYER: approx = one_based >= 2 && (one_based - 2) % 4 == 0; break;
+        case GACONV_SCHED_ALT_LAYER_ALT_BATCH: approx = one_based % 2 == 0 && step % 2 == 1; break;
+        case GACONV_SCHED_ALL_LAYERS_EVERY_4TH_BATCH: approx = step % 4 == 3; break;
+        case GACONV_SCHED_LAYER2_ALT_BATCH: approx = one_based == 2 && step % 2 == 1; break;
+        case GACONV_SCHED_SEEDED_FRACTION_ALT_BATCH: approx = step % 2 == 1 && s->mask[layer]; break;
+    }
+    return approx ? s->method : GACONV_METHOD_EXACT;
+}
+
+gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t* s, int32_t layer, int64_t step, const void* x,
+                                          const void* dy, float* dw, const gaconv_conv_desc_t* desc, void* stream)
+{
+    const int32_t m = gaconv_schedule_method(s, layer, step);
+    if (m == -2) return GACONV_ERR_BAD_DESC;
+    if (m == GACONV_METHOD_EXACT) return gaconv_dw_exact(x, dy, dw, desc, stream);
+    const uint64_t seed = splitmix64(s->seed ^ splitmix64((uint64_t)step * 0x100000001B3ull + (uint64_t)layer));
+    return gaconv_dw_approx(m, x, dy, dw, desc, seed, stream);
+}
+
+void gaconv_schedule_destroy(gaconv_schedule_t* s)
+{
+    if (s == nullptr) return;
+    delete[] s->mask;
+    delete s;
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+// Zero gradient (paper Section 2.1) and random gradient (Section 2.2).
+//
+// Random gradient: independent N(0, std^2) values from a counter-based generator, so that a value
+// depends only on (seed, element index) and a new seed per batch regenerates everything:
+//   Philox-4x32-10 (Salmon et al., SC'11), key = (seed low, seed high), counter = (j,0,0,0)
+//   -> words w0..w3 -> elements 4j..4j+3 by Box-Muller:
+//   u1 = (w_a+1) 2^-32, u2 = w_b 2^-32, rho = sqrt(-2 ln u1), (rho cos 2 pi u2, rho sin 2 pi u2)
+// for the pairs (w0,w1) and (w2,w3).  Element i is position i of the logical [k][c][r][s] order.
+#include "gaconv_internal.h"
+
+namespace gaconv {
+namespace {
+
+__global__ void __launch_bounds__(256) zero_kernel(float* __restrict__ dw, size_t count)
+{
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    const size_t nvec = count / 4;
+    float4* v = reinterpret_cast<float4*>(dw);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride)
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (size_t i = nvec * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) dw[i] = 0.f;
+}
+
+__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1)
+{
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+    const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+}
+
+__device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float& z0, float& z1)
+{
+    // ln in double: u1 close to 1 would lose all its information in fp32
+    const double u1 = ((double)wa + 1.0) * (1.0 / 4294967296.0);
+    const float rho = sqrtf((float)(-2.0 * log(u1)));
+    float sn, cs;
+    sincospif(2.0f * ((float)wb * (1.0f / 4294967296.0f)), &sn, &cs);
+    z0 = rho * cs; z1 = rho * sn;
+}
+
+__global__ void __launch_bounds__(256)
+random_kernel(float* __restrict__ dw, size_t count, Geom g, uint32_t key0, uint32_t key1, float std, bool contiguous)
+{
+    const size_t j = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (4 * j >= count) return;
+    uint32_t c[4] = {(uint32_t)j, 0u, 0u, 0u};
+    uint32_t k0 = key0, k1 = key1;
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        philox_round(c, k0, k1);
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    float z[4];
+    box_muller(c[0], c[1], z[0], z[1]);
+    box_muller(c[2], c[3], z[2], z[3]);
+    if (contiguous && 4 * j + 3 < count) {
+        reinterpret_cast<float4*>(dw)[j] = make_float4(std * z[0], std * z[1], std * z[2], std * z[3]);
+        return;
+    }
+    for (int t = 0; t < 4; ++t) {
+        const size_t i = 4 * j + t;
+        if (i >= count) break;
+        // logical [k][c][r][s] position of element i -> offset in the chosen dW layout
+        const int s = (int)(i % g.s); size_t rest = i / g.s;
+        const int r = (int)(rest % g.r); rest /= g.r;
+        const int cc = (int)(rest % g.c); const int k = (int)(rest / g.c);
+        dw[k * g.ws_k + cc * g.ws_c + r * g.ws_r + s * g.ws_s] = std * z[t];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream)
+{
+    size_t blocks = (count / 4 + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    zero_kernel<<<(unsigned)blocks, 256, 0, stream>>>(dw, count);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cudaStream_t stream)
+{
+    const size_t count = (size_t)g.k * g.c * g.r * g.s;
+    const size_t threads = (count + 3) / 4;
+    const bool contiguous = (g.ws_s == 1 && g.ws_r == g.s && g.ws_c == (long long)g.r * g.s);
+    random_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(dw, count, g, (uint32_t)seed,
+                                                                          (uint32_t)(seed >> 32), std, contiguous);
+    return cudaGetLastError();
+}
+
+}  // namespace gaconv

@@ -1,0 +1,64 @@
+// Internal declarations shared by the translation units of libgaconv (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "gaconv.h"
+
+namespace gaconv {
+
+// ---- workspace layout -------------------------------------------------------------------------
+// [0, 256)            control: word 0 = sticky device status (0 ok, 1 bounded wait gave up)
+// [256, 256+16 KiB)   ticket counters, all zero between calls (each kernel resets what it used)
+// [kWsDataOffset, ..) per-call data (selection results, split partials)
+constexpr size_t kWsCounterOffset = 256;
+constexpr int    kWsNumCounters   = 4096;
+constexpr size_t kWsDataOffset    = kWsCounterOffset + sizeof(uint32_t) * kWsNumCounters;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Geometry with derived sizes and element strides of the chosen layouts.
+struct Geom {
+    int n, c, h, w, k, r, s, p, q;
+    int stride_h, stride_w, pad_h, pad_w;
+    long long xs_n, xs_c, xs_h, xs_w;   // element strides of X
+    long long ws_k, ws_c, ws_r, ws_s;   // element strides of dW
+    bool bf16;
+    float alpha;
+};
+
+// ---- selection (Algorithm 1, arg-max and sum lines) ----
+cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_sparse, const Geom& g,
+                          cudaStream_t stream);
+
+// ---- gather-accumulate (Algorithm 1, patch accumulation line) ----
+struct GatherPlan {
+    int chunks;          // CTAs per output channel, each owning a contiguous range of images
+    int imgs_per_chunk;
+    size_t partial_bytes;
+};
+GatherPlan plan_gather(const Geom& g);
+cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, float* dw, float* partial,
+                          uint32_t* counters, const Geom& g, const GatherPlan& plan, cudaStream_t stream);
+
+// ---- zero / random gradient ----
+cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream);
+cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cudaStream_t stream);
+
+// ---- exact filter gradient, direct FP32 kernel (any shape, any layout) ----
+struct DirectPlan {
+    int tiles_k, tiles_c;   // output tiles of 16 x 16 (k x c), all (r,s) per tile
+    int bp, bq;             // output-pixel band handled per work item
+    int bands_p, bands_q;
+    int items;              // n * bands_p * bands_q
+    int splits;             // CTAs per output tile along the reduction
+    size_t partial_bytes;
+    bool tiled;             // false: filter size without a tiled instantiation -> per-element kernel
+};
+DirectPlan plan_direct(const Geom& g);
+cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
+                          const Geom& g, const DirectPlan& plan, cudaStream_t stream);
+
+}  // namespace gaconv

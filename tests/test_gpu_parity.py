@@ -1,0 +1,238 @@
+"""Parity of the CUDA path (through the C ABI) with the oracle, element by element, on seeded inputs.
+
+Tolerances: selection indices bit-exact; fp32 inputs within 1e-5 and bf16 inputs within 2e-2 of the
+sum of |products| per output element; selection sums within 1e-6 of sum |dY| of the map."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_1908_05460_b200 import binding as B
+from paper_1908_05460_b200 import inputs as I
+from paper_1908_05460_b200.layers import ConvLayer, config1_layer, resnet20_layers, vgg19_layers, cnn2_layers
+from helpers import GpuLayer, norm_err, oshape, to_f64, TOL_F32, TOL_BF16, TOL_SUM
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = [torch.float32, torch.bfloat16]
+
+
+def tol(dtype):
+    return TOL_F32 if dtype == torch.float32 else TOL_BF16
+
+
+# small cases spanning several tiles with ragged tails: C=3, W=2, stride 2, 5x5, odd sizes
+SMALL = [
+    config1_layer(),
+    ConvLayer("c3 stem", 5, 3, 32, 32, 16, 3, 3, 1, 1, dy_std=1.0),
+    ConvLayer("stride2", 6, 16, 32, 32, 32, 3, 3, 2, 1),
+    ConvLayer("5x5", 4, 3, 32, 32, 64, 5, 5, 1, 2, x_dist="uniform_pm1"),
+    ConvLayer("5x5 c64", 3, 64, 16, 16, 64, 5, 5, 1, 2),
+    ConvLayer("ragged", 3, 19, 13, 11, 21, 3, 3, 1, 1, dy_std=1.0),
+    ConvLayer("ragged s2 nopad", 2, 7, 15, 9, 5, 3, 3, 2, 0, dy_std=1.0),
+    ConvLayer("w2", 9, 40, 2, 2, 24, 3, 3, 1, 1),
+    ConvLayer("4x4", 8, 48, 4, 4, 80, 3, 3, 1, 1),
+    ConvLayer("8x8", 8, 64, 8, 8, 64, 3, 3, 1, 1),
+    ConvLayer("1x1", 4, 20, 9, 9, 12, 1, 1, 1, 0, dy_std=1.0),
+    ConvLayer("7x7 filter", 2, 5, 12, 12, 6, 7, 7, 1, 3, dy_std=1.0),
+    ConvLayer("one image one channel", 1, 1, 5, 5, 1, 3, 3, 1, 1, dy_std=1.0),
+]
+
+
+def _inputs(layer, dtype, tag):
+    return I.make_layer_inputs(layer, dtype, config=9, layer_index=tag)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("li", range(len(SMALL)), ids=[l.name for l in SMALL])
+def test_exact_matches_oracle(li, dtype):
+    layer = SMALL[li]
+    x, dy = _inputs(layer, dtype, li)
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.5)
+    g = GpuLayer(layer, dtype, x, dy, alpha=0.5)
+    assert norm_err(g.exact(), ref, dn) <= tol(dtype)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("li", range(len(SMALL)), ids=[l.name for l in SMALL])
+def test_top1_matches_oracle(li, dtype):
+    layer = SMALL[li]
+    x, dy = _inputs(layer, dtype, li)
+    xd, dyd = to_f64(x), to_f64(dy)
+    idx_ref, sum_ref, abs_ref = oracle.top1_select(dyd)
+    ref, dn = oracle.dw_top1(xd, dyd, oshape(layer), 1.0 / 128)
+    g = GpuLayer(layer, dtype, x, dy, alpha=1.0 / 128)
+    idx, s, sparse = g.select(want_sparse=True)
+    np.testing.assert_array_equal(idx, idx_ref)                       # bit-exact selection
+    assert np.max(np.abs(s - sum_ref) / np.maximum(abs_ref, 1e-300)) <= TOL_SUM
+    # the dense sparse tensor: the (rounded) sum at the selected position, zero elsewhere
+    sp = sparse.to(torch.float64).numpy().reshape(layer.n, layer.k, -1)
+    want = np.zeros_like(sp)
+    np.put_along_axis(want, idx_ref[..., None].astype(np.int64),
+                      torch.from_numpy(s).to(dtype).to(torch.float64).numpy()[..., None], axis=2)
+    np.testing.assert_array_equal(sp, want)
+    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
+
+
+@pytest.mark.parametrize("x_layout,dw_layout", [(B.X_NCHW, B.DW_KCRS), (B.X_NHWC, B.DW_KCRS), (B.X_NCHW, B.DW_KRSC)])
+def test_other_layouts(x_layout, dw_layout):
+    layer = SMALL[5]
+    x, dy = _inputs(layer, torch.float32, 40)
+    xd, dyd = to_f64(x), to_f64(dy)
+    g = GpuLayer(layer, torch.float32, x, dy, x_layout=x_layout, dw_layout=dw_layout)
+    ref, dn = oracle.dw_exact(xd, dyd, oshape(layer))
+    assert norm_err(g.exact(), ref, dn) <= TOL_F32
+    ref, dn = oracle.dw_top1(xd, dyd, oshape(layer))
+    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= TOL_F32
+    z = oracle.dw_random(ref.size, 5, 0.25).reshape(ref.shape)
+    assert np.max(np.abs(g.approx(B.METHOD_RANDOM, seed=5) * (0.25 * 128) - z)) < 1e-5 * 0.25 * 8
+
+
+def test_selection_ties_and_planted_maxima():
+    layer = ConvLayer("ties", 4, 2, 32, 32, 8, 3, 3, 1, 1)
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 50)
+        dy = dy.clone()
+        dy[0, 0].zero_()                                   # all-zero map -> index 0
+        dy[0, 1, 31, 31] = 64.0; dy[0, 1, 3, 7] = -64.0    # equal magnitudes -> the earlier one
+        dy[1, 2, 0, 0] = -77.0                             # first element
+        dy[1, 3, 31, 31] = 77.0                            # last element
+        dy[2, 4] = 1.0                                     # constant map -> index 0
+        dy[3, 5, 10, :] = -3.0                             # a row of equal maxima -> its first
+        g = GpuLayer(layer, dtype, x, dy)
+        idx, s, _ = g.select()
+        idx_ref, sum_ref, abs_ref = oracle.top1_select(to_f64(dy))
+        np.testing.assert_array_equal(idx, idx_ref)
+        assert idx[0, 0] == 0 and idx[0, 1] == 3 * 32 + 7 and idx[1, 2] == 0 and idx[1, 3] == 1023
+        assert idx[2, 4] == 0 and idx[3, 5] == 320
+        assert np.max(np.abs(s - sum_ref) / np.maximum(abs_ref, 1e-30)) <= TOL_SUM
+
+
+def test_bf16_ties_occur_naturally_and_match():
+    """bf16 gradients collide often; the tie rule is exercised on plain random inputs too."""
+    layer = ConvLayer("bf16 ties", 64, 4, 32, 32, 32, 3, 3, 1, 1)
+    _, dy = _inputs(layer, torch.bfloat16, 51)
+    d = to_f64(dy).reshape(layer.n * layer.k, -1)
+    top2 = np.sort(np.abs(d), axis=1)[:, -2:]
+    assert np.count_nonzero(top2[:, 0] == top2[:, 1]) >= 5
+    g = GpuLayer(layer, torch.bfloat16, torch.zeros(layer.n, layer.c, layer.h, layer.w, dtype=torch.bfloat16), dy)
+    np.testing.assert_array_equal(g.select()[0], oracle.top1_select(to_f64(dy))[0])
+
+
+def test_zero_and_random_methods():
+    layer = config1_layer()
+    x, dy = _inputs(layer, torch.float32, 60)
+    g = GpuLayer(layer, torch.float32, x, dy, rand_std=1.0 / 128)
+    z = g.approx(B.METHOD_ZERO)
+    assert np.all(z == 0) and not np.any(np.signbit(z))
+    count = z.size
+    for seed in (0, 1, 0xDEADBEEFCAFEF00D):
+        got = g.approx(B.METHOD_RANDOM, seed=seed).reshape(-1)
+        ref = oracle.dw_random(count, seed, 1.0 / 128)
+        assert np.max(np.abs(got - ref) / ((1.0 / 128) * np.maximum(1.0, np.abs(ref) * 128))) <= 1e-5
+    # a count that is not a multiple of four, written through the strided (KRSC) path
+    odd = ConvLayer("odd", 1, 3, 5, 5, 5, 3, 3, 1, 1)
+    xo, dyo = _inputs(odd, torch.float32, 61)
+    go = GpuLayer(odd, torch.float32, xo, dyo, rand_std=2.0)
+    got = go.approx(B.METHOD_RANDOM, seed=9).reshape(-1)
+    assert np.max(np.abs(got - oracle.dw_random(got.size, 9, 2.0))) <= 1e-5 * 2.0 * 6
+    big = ConvLayer("big", 1, 256, 4, 4, 256, 3, 3, 1, 1)
+    gb = GpuLayer(big, torch.float32, torch.zeros(1, 256, 4, 4), torch.zeros(1, 256, 4, 4), dw_layout=B.DW_KCRS)
+    v = gb.approx(B.METHOD_RANDOM, seed=77).reshape(-1) * 128
+    assert abs(v.mean()) < 4 / np.sqrt(v.size) and abs(v.std() - 1) < 0.01
+
+
+def test_runs_are_bitwise_reproducible():
+    layer = SMALL[2]
+    x, dy = _inputs(layer, torch.bfloat16, 70)
+    g = GpuLayer(layer, torch.bfloat16, x, dy)
+    a, b = g.exact(), g.exact()
+    np.testing.assert_array_equal(a, b)
+    a, b = g.approx(B.METHOD_TOP1), g.approx(B.METHOD_TOP1)
+    np.testing.assert_array_equal(a, b)
+
+
+def test_full_selection_invariant_on_gpu():
+    """With one output pixel per map the top-1 method keeps everything, so it must equal exact dW."""
+    layer = ConvLayer("p=q=1", 16, 8, 3, 3, 8, 3, 3, 1, 0, dy_std=1.0)
+    x, dy = _inputs(layer, torch.float32, 71)
+    g = GpuLayer(layer, torch.float32, x, dy)
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer))
+    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= TOL_F32
+    assert norm_err(g.exact(), ref, dn) <= TOL_F32
+
+
+def test_from_host_entry_point():
+    layer = config1_layer()
+    x, dy = _inputs(layer, torch.float32, 72)
+    g = GpuLayer(layer, torch.float32, x, dy)
+    xh = I.to_nhwc(x).pin_memory(); dyh = dy.contiguous().pin_memory()
+    out = torch.empty(layer.k, layer.r, layer.s, layer.c, dtype=torch.float32).pin_memory()
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer))
+    g.x.zero_(); g.dy.zero_()
+    B.gaconv_dw_from_host(B.METHOD_EXACT, xh, dyh, out, g.x, g.dy, g.dw, g.desc)
+    assert norm_err(I.krsc_to_kcrs(out).to(torch.float64).numpy(), ref, dn) <= TOL_F32
+    ref, dn = oracle.dw_top1(to_f64(x), to_f64(dy), oshape(layer))
+    B.gaconv_dw_from_host(B.METHOD_TOP1, xh, dyh, out, g.x, g.dy, g.dw, g.desc)
+    assert norm_err(I.krsc_to_kcrs(out).to(torch.float64).numpy(), ref, dn) <= TOL_F32
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+
+
+def test_schedule_run_layer_dispatches_the_scheduled_method():
+    layer = config1_layer()
+    x, dy = _inputs(layer, torch.float32, 73)
+    g = GpuLayer(layer, torch.float32, x, dy)
+    ref_e, dn_e = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer))
+    ref_t, dn_t = oracle.dw_top1(to_f64(x), to_f64(dy), oshape(layer))
+    s = B.Schedule(2, B.SCHED_LAYER2_ALT_BATCH, B.METHOD_TOP1)
+    for step in range(4):
+        for l in range(2):
+            g.dw.fill_(float("nan"))
+            s.run_layer(l, step, g.x, g.dy, g.dw, g.desc)
+            if l == 1 and step % 2 == 1:
+                assert norm_err(g.logical_dw(), ref_t, dn_t) <= TOL_F32
+            else:
+                assert norm_err(g.logical_dw(), ref_e, dn_e) <= TOL_F32
+    r = B.Schedule(3, B.SCHED_ALL_LAYERS_EVERY_4TH_BATCH, B.METHOD_RANDOM, seed=5)
+    r.run_layer(0, 3, g.x, g.dy, g.dw, g.desc); a = g.logical_dw()
+    r.run_layer(0, 7, g.x, g.dy, g.dw, g.desc); b = g.logical_dw()
+    r.run_layer(1, 7, g.x, g.dy, g.dw, g.desc); c = g.logical_dw()
+    assert abs(np.corrcoef(a.ravel(), b.ravel())[0, 1]) < 0.1 and abs(np.corrcoef(b.ravel(), c.ravel())[0, 1]) < 0.1
+    assert abs(a.std() * 128 - 1) < 0.1
+
+
+# ---- full-size layers in the configuration the benchmark times: sampled outputs + whole top-1 ----
+FULL = [("resnet", 1), ("resnet", 7), ("resnet", 13), ("resnet", 18), ("vgg", 1), ("vgg", 5), ("vgg", 9), ("vgg", 15),
+        ("cnn", 0), ("cnn", 1)]
+
+
+@pytest.mark.parametrize("net,li", FULL, ids=["%s%d" % f for f in FULL])
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+def test_full_size_layers(net, li, dtype):
+    layer = {"resnet": resnet20_layers, "vgg": vgg19_layers, "cnn": cnn2_layers}[net](128)[li]
+    if dtype == torch.float32 and net == "vgg":
+        pytest.skip("VGG-19 workload is bf16 only")
+    cfg = {"resnet": 2, "cnn": 3, "vgg": 4}[net]
+    x, dy = I.make_layer_inputs(layer, dtype, cfg, li)
+    xd, dyd = to_f64(x), to_f64(dy)
+    g = GpuLayer(layer, dtype, x, dy)
+    sh = oshape(layer)
+    # top-1: the oracle covers the whole layer
+    idx, s, _ = g.select()
+    idx_ref, sum_ref, abs_ref = oracle.top1_select(dyd)
+    np.testing.assert_array_equal(idx, idx_ref)
+    assert np.max(np.abs(s - sum_ref) / abs_ref) <= TOL_SUM
+    ref, dn = oracle.dw_top1(xd, dyd, sh)
+    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
+    # exact: sampled output elements, each computed by the oracle on its own
+    got = g.exact()
+    rng = np.random.default_rng(li)
+    picks = {(0, 0, 0, 0), (layer.k - 1, layer.c - 1, layer.r - 1, layer.s - 1), (layer.k - 1, 0, 0, layer.s - 1)}
+    while len(picks) < 48:
+        picks.add((int(rng.integers(layer.k)), int(rng.integers(layer.c)), int(rng.integers(layer.r)), int(rng.integers(layer.s))))
+    worst = 0.0
+    for (k, c, r, s_) in picks:
+        v, nrm = oracle.dw_exact_at(xd, dyd, sh, k, c, r, s_)
+        worst = max(worst, abs(got[k, c, r, s_] - v) / nrm)
+    assert worst <= tol(dtype)
+    assert np.all(np.isfinite(got))
