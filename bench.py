@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the filter-gradient (dW) hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic batch of a layer set (default: the 19
+convolutions of ResNet-20 for CIFAR-10 at batch 128, inputs in bf16 and in fp32): for every layer the
+exact dW, the top-1 approximation (Algorithm 1), the zero gradient and the random gradient, each
+dispatched by the approximation-schedule driver.  The step is captured once in a CUDA graph and
+replayed; it is ordered method-major so that a buffer is touched again only after more than twice
+the L2 capacity of other data has streamed through (cold-L2 protocol).
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per layer pass (all four methods of one
+layer in one dtype), aggregated over GPUs: step time / (layer passes per step * n_gpus).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dW-conv us/layer"
+UNIT = "us/layer"
+WORKLOADS = {2: "resnet20_cifar10_n128", 3: "cnn2_cifar10_n128", 4: "vgg19_cifar10_n128"}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.path)
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = mx
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+def oracle_sample_us_per_layer(layers, imgs: int):
+    """Times the oracle (exact + top-1 + zero + random) on `imgs` images of every distinct layer shape
+    and extrapolates linearly in the batch size.  Returns (us per layer pass, seconds spent, threads)."""
+    import numpy as np
+    from oracle import oracle
+    from paper_1908_05460_b200 import inputs as I
+    import torch
+    seen, total_us, spent = {}, 0.0, 0.0
+    for li, l in enumerate(layers):
+        key = (l.c, l.k, l.h, l.r, l.stride)
+        if key not in seen:
+            ls = l.with_batch(min(imgs, l.n))
+            x, dy = I.make_layer_inputs(ls, torch.float32, 2, li)
+            xd, dyd = x.double().numpy(), dy.double().numpy()
+            sh = oracle.Shape(ls.n, ls.c, ls.h, ls.w, ls.k, ls.r, ls.s, ls.stride, ls.stride, ls.pad, ls.pad)
+            t0 = time.perf_counter()
+            oracle.dw_exact(xd, dyd, sh)
+            oracle.dw_top1(xd, dyd, sh)
+            t1 = time.perf_counter()
+            cnt = l.k * l.c * l.r * l.s
+            oracle.dw_zero(cnt); oracle.dw_random(cnt, 1, 1.0 / 128)
+            t2 = time.perf_counter()
+            seen[key] = ((t1 - t0) * (l.n / ls.n) + (t2 - t1)) * 1e6
+            spent += t2 - t0
+        total_us += seen[key]
+    return total_us / len(layers), spent, oracle.num_threads()
+
+
+def run_reference(args, layers):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(args.warmup):
+        oracle_sample_us_per_layer(layers, 1)
+    vals, t0 = [], time.perf_counter()
+    threads = 1
+    for _ in range(args.steps):
+        v, _, threads = oracle_sample_us_per_layer(layers, 1)
+        vals.append(v)
+    wall = time.perf_counter() - t0
+    value = statistics.mean(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / args.steps * 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOADS[args.config], "note": "CPU oracle; each step times 1 of 128 images per "
+                       "distinct layer shape and scales by the batch size"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": "1 of 128 images per distinct layer shape, exact+top1+zero+random, x128"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4], help="layer set: 2 ResNet-20, 3 two-layer CNN, 4 VGG-19")
+    ap.add_argument("--batch", type=int, default=128)
+    ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
+    ap.add_argument("--layer-iters", type=int, default=10, help="cold per-layer timing iterations")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--detail", default=None, help="write the per-layer table to this JSON file")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_1908_05460_b200.layers import layer_set
+    layers = layer_set(args.config, args.batch)
+    if args.impl == "reference":
+        run_reference(args, layers)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1908_05460_b200 import binding as B
+    from paper_1908_05460_b200 import inputs as I
+    from paper_1908_05460_b200 import build as build_mod
+
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        build_mod.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    B.load()
+    peaks = measured_peaks()
+
+    dtype_names = (args.dtypes.split(",") if args.dtypes else (["bf16"] if args.config == 4 else ["bf16", "f32"]))
+    dtypes = [{"bf16": torch.bfloat16, "f32": torch.float32}[d] for d in dtype_names]
+
+    # ---- inputs: generated on the host (seeded), resident in HBM before any timed region ----
+    class Slot:
+        pass
+    slots = []
+    h2d = d2h = 0
+    for dt, dname in zip(dtypes, dtype_names):
+        for li, l in enumerate(layers):
+            s = Slot()
+            s.layer, s.li, s.dtype, s.dname = l, li, dt, dname
+            x, dy = I.make_layer_inputs(l, dt, args.config, li + 1000 * rank)
+            s.x_host = I.to_nhwc(x).pin_memory(); s.dy_host = dy.contiguous().pin_memory()
+            s.x = s.x_host.cuda(); s.dy = s.dy_host.cuda()
+            s.dw = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32, device="cuda")
+            s.dw_host = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32).pin_memory()
+            s.desc = B.make_desc(l, dt, alpha=1.0 / l.n)
+            s.ws = B.attach_workspace(s.desc)
+            s.eb = 2 if dt == torch.bfloat16 else 4
+            h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs
+            d2h += 4 * s.dw.numel() * 4
+            slots.append(s)
+    L = len(layers)
+    input_bytes = sum((s.x.numel() + s.dy.numel()) * s.eb for s in slots)
+
+    methods = [("exact", B.METHOD_EXACT), ("top1", B.METHOD_TOP1), ("zero", B.METHOD_ZERO), ("random", B.METHOD_RANDOM)]
+    # schedule 3 of the paper (all layers every 4th batch): step 4t+3 approximates, others are exact
+    scheds = {m: B.Schedule(L, B.SCHED_ALL_LAYERS_EVERY_4TH_BATCH, m if m >= 0 else B.METHOD_TOP1, 0.0, 1234)
+              for _, m in methods}
+
+    def run_one(s, m, t):
+        scheds[m].run_layer(s.li, 4 * t + (3 if m >= 0 else 0), s.x, s.dy, s.dw, s.desc)
+
+    def step(t):
+        for _, m in methods:                # method-major: a buffer is reused only after a full input pass
+            for s in slots:
+                run_one(s, m, t)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up, graph capture ----
+    c0 = B.gaconv_launch_count()
+    step(0)
+    launches_per_step = B.gaconv_launch_count() - c0
+    torch.cuda.synchronize()
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(1)
+    run_step = (lambda t: graph.replay()) if graph is not None else step
+    for t in range(args.warmup):
+        run_step(t)
+    barrier()
+
+    # ---- timed region: exactly K steps ----
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for t in range(args.steps):
+        run_step(t)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    if rank == 0:
+        time.sleep(0.2)
+    clocks = sampler.stop() if rank == 0 else None
+    tt = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms_step = float(tt.item()) / args.steps
+    passes = len(slots)
+    value = ms_step * 1e3 / (passes * world)
+
+    # ---- per-layer cold timing (L2 flushed before every launch), on the launching stream ----
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def cold_us(fn, iters):
+        ts = []
+        for _ in range(iters):
+            flush.fill_(1)
+            es.record(); fn(); ee.record()
+            ee.synchronize()
+            ts.append(es.elapsed_time(ee) * 1e3)
+        return statistics.median(ts)
+
+    empty_pair_us = cold_us(lambda: None, 20)
+    table = []
+    for s in slots:
+        row = {"layer": s.layer.name, "index": s.li, "dtype": s.dname}
+        for name, m in methods:
+            row[name + "_us"] = cold_us(lambda: run_one(s, m, 2), args.layer_iters)
+        l = s.layer
+        fl, be, bt = l.flops_exact(), l.bytes_exact(s.eb), l.bytes_top1(s.eb)
+        t_tensor = fl / (peaks["bf16_tflops"] * 1e12 * (1.0 if s.eb == 2 else 0.5)) * 1e6   # tf32 nominal ratio 1/2
+        t_hbm = be / (peaks["hbm_gbs"] * 1e9) * 1e6
+        row.update({"gflop": fl / 1e9, "exact_bytes": be, "top1_bytes": bt,
+                    "exact_tflops": fl / row["exact_us"] / 1e6, "exact_gbs": be / row["exact_us"] / 1e3,
+                    "exact_roof_us": max(t_tensor, t_hbm), "exact_bound": "tensor" if t_tensor > t_hbm else "hbm",
+                    "exact_frac": max(t_tensor, t_hbm) / row["exact_us"],
+                    "top1_gbs": bt / row["top1_us"] / 1e3, "top1_frac": bt / (peaks["hbm_gbs"] * 1e3) / row["top1_us"],
+                    "top1_speedup": row["exact_us"] / row["top1_us"]})
+        table.append(row)
+    sum_us = {name: sum(r[name + "_us"] for r in table) for name, _ in methods}
+
+    # ---- roofline of the dominant kernel family (largest share of the cold per-layer time) ----
+    fam = max(("exact", "top1"), key=lambda n: sum_us[n])
+    if fam == "exact":
+        hb = [r for r in table if r["exact_bound"] == "hbm"]; tb = [r for r in table if r["exact_bound"] == "tensor"]
+        if sum(r["exact_us"] for r in hb) >= sum(r["exact_us"] for r in tb):
+            ach = sum(r["exact_bytes"] for r in hb) / sum(r["exact_us"] for r in hb) / 1e3
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "kernel": "exact dW",
+                    "launches": len(hb)}
+        else:
+            ach = sum(r["gflop"] for r in tb) / sum(r["exact_us"] for r in tb) / 1e3
+            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "kernel": "exact dW", "launches": len(tb)}
+    else:
+        ach = sum(r["top1_bytes"] for r in table) / sum_us["top1"] / 1e3
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "kernel": "top-1 select+gather", "launches": len(table)}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = peaks["source"]
+    roof["traffic"] = None
+
+    # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step(t):
+            for _, m in methods:
+                for s in slots:
+                    B.gaconv_dw_from_host(m, s.x_host, s.dy_host, s.dw_host, s.x, s.dy, s.dw, s.desc, seed=t)
+        e2e_step(0)
+        barrier()
+        k2 = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        ev0.record()
+        for t in range(k2):
+            e2e_step(t)
+        ev1.record()
+        barrier()
+        ms_e = torch.tensor([ev0.elapsed_time(ev1) / k2], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(ms_e, op=dist.ReduceOp.MAX)
+        e2e = {"value": float(ms_e.item()) * 1e3 / (passes * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": k2}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if not args.no_cpu:
+        imgs, spent = 1, 0.0
+        v, spent, threads = oracle_sample_us_per_layer(layers, imgs)
+        while spent < 6.0 and imgs < args.batch:
+            imgs *= 4
+            v, spent, threads = oracle_sample_us_per_layer(layers, imgs)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "%d of %d images per distinct layer shape (exact+top1+zero+random, fp64), scaled to the "
+                         "full batch; %.1f s of CPU work" % (min(imgs, args.batch), args.batch, spent)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "+".join(dtype_names) + " inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "%s (%d conv layers x {%s} x {exact, top1, zero, random})"
+                               % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), L, ",".join(dtype_names)),
+                   "layer_passes_per_step": passes, "cuda_graph": graph is not None,
+                   "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
+                         "order); per-layer timings flush L2 with a 256 MB write before every launch" % (input_bytes / 1e6)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roof, "cpu_baseline": cpu,
+        "breakdown_us": {"cold_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
+                         "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
+                         "top1_speedup_over_exact": sum_us["exact"] / sum_us["top1"]},
+        "paper_context": "paper reports >7% training wall-clock speedup (ResNet-20/VGG-19, Titan Xp, TF 1.13, cuDNN 7.4.2)",
+    }
+    if args.detail:
+        os.makedirs(os.path.dirname(os.path.abspath(args.detail)), exist_ok=True)
+        json.dump({"summary": line, "layers": table}, open(args.detail, "w"), indent=1)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -73,6 +73,10 @@ typedef struct gaconv_conv_desc {
 
 const char *gaconv_status_string(gaconv_status_t status);
 
+/* Number of kernels this library has enqueued since it was loaded (all threads).  Bookkeeping for
+ * benchmarks; no counterpart in the paper. */
+uint64_t gaconv_launch_count(void);
+
 /* Device scratch one call needs for `method` (GACONV_METHOD_EXACT for the exact path) with this
  * descriptor (its workspace fields are ignored).  Never fails for a valid descriptor; *bytes > 0. */
 gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t *desc, int32_t method, size_t *bytes);

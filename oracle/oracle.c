@@ -288,3 +288,11 @@ void oracle_dw_random(double *dw, size_t count, uint64_t seed, double std)
         for (int t = 0; t < 4 && 4 * j + t < count; ++t) dw[4 * j + t] = std * z[t];
     }
 }
+
+/* Number of OpenMP threads the exact path uses (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_num_threads(void) { return 1; }
+#endif

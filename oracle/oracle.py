@@ -177,3 +177,7 @@ def dw_random(count: int, seed: int, std: float):
     out = np.empty(count)
     lib().oracle_dw_random(_d(out), ctypes.c_size_t(count), ctypes.c_uint64(seed), ctypes.c_double(std))
     return out
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())

@@ -29,7 +29,7 @@ SCHED_EVERY_4TH_LAYER, SCHED_ALT_LAYER_ALT_BATCH, SCHED_ALL_LAYERS_EVERY_4TH_BAT
     SCHED_SEEDED_FRACTION_ALT_BATCH = range(5)
 
 EXPORTS = [
-    "gaconv_status_string", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
+    "gaconv_status_string", "gaconv_launch_count", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
     "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_poll_async_status",
     "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_destroy",
 ]
@@ -65,6 +65,8 @@ def load():
     dp = ctypes.POINTER(ConvDesc)
     lib.gaconv_status_string.restype = ctypes.c_char_p
     lib.gaconv_status_string.argtypes = [ctypes.c_int]
+    lib.gaconv_launch_count.restype = ctypes.c_uint64
+    lib.gaconv_launch_count.argtypes = []
     lib.gaconv_workspace_size.argtypes = [dp, i32, ctypes.POINTER(sz)]
     lib.gaconv_workspace_init.argtypes = [vp, sz, vp]
     lib.gaconv_dw_exact.argtypes = [vp, vp, vp, dp, vp]
@@ -84,6 +86,10 @@ def load():
 
 def status_string(status: int) -> str:
     return load().gaconv_status_string(status).decode()
+
+
+def gaconv_launch_count() -> int:
+    return int(load().gaconv_launch_count())
 
 
 def _check(status: int, where: str):

@@ -1,11 +1,15 @@
 // C-ABI entry points of libgaconv: argument validation, workspace planning, kernel dispatch and the
 // approximation-schedule driver (paper Section 2.5).  Every step of the path runs in this library's
 // kernels; there is no CPU or library fallback.
+#include <atomic>
 #include <new>
 
 #include "gaconv_internal.h"
 
 using namespace gaconv;
+
+static std::atomic<uint64_t> g_launches{0};
+void gaconv::note_launch(int count) { g_launches.fetch_add((uint64_t)count, std::memory_order_relaxed); }
 
 namespace {
 
@@ -110,6 +114,8 @@ const char* gaconv_status_string(gaconv_status_t s)
     }
     return "unknown status";
 }
+
+uint64_t gaconv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t method, size_t* bytes)
 {

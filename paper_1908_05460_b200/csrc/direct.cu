@@ -137,6 +137,7 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_
     if (!pl.tiled) {
         const long long total = (long long)g.k * g.r * g.s * g.c;
         direct_element_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(x, dy, dw, g);
+        note_launch();
         return cudaGetLastError();
     }
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
@@ -145,6 +146,7 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_
 #define GACONV_DIRECT_CASE(RR, SS)                                                                         \
     if (g.r == RR && g.s == SS) {                                                                          \
         direct_tiled_kernel<T, RR, SS><<<grid, 256, smem, stream>>>(x, dy, dw, partial, counters, g, pl); \
+        note_launch();                                                                                     \
         return cudaGetLastError();                                                                         \
     }
     GACONV_DIRECT_CASE(1, 1)

@@ -77,6 +77,7 @@ cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream)
     if (blocks < 1) blocks = 1;
     if (blocks > 148 * 8) blocks = 148 * 8;
     zero_kernel<<<(unsigned)blocks, 256, 0, stream>>>(dw, count);
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -87,6 +88,7 @@ cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cu
     const bool contiguous = (g.ws_s == 1 && g.ws_r == g.s && g.ws_c == (long long)g.r * g.s);
     random_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(dw, count, g, (uint32_t)seed,
                                                                           (uint32_t)(seed >> 32), std, contiguous);
+    note_launch();
     return cudaGetLastError();
 }
 

@@ -17,6 +17,8 @@ constexpr size_t kWsCounterOffset = 256;
 constexpr int    kWsNumCounters   = 4096;
 constexpr size_t kWsDataOffset    = kWsCounterOffset + sizeof(uint32_t) * kWsNumCounters;
 
+void note_launch(int count = 1);   // bookkeeping behind gaconv_launch_count()
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Geometry with derived sizes and element strides of the chosen layouts.

@@ -208,6 +208,7 @@ cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_spa
         if (vec) select_kernel<float, true><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
         else     select_kernel<float, false><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
     }
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -237,6 +238,7 @@ cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, f
     else
         gather_kernel<float><<<grid, 256, smem, stream>>>(static_cast<const float*>(x), idx, sum, dw, partial,
                                                           counters, g, plan.chunks, plan.imgs_per_chunk);
+    note_launch();
     return cudaGetLastError();
 }
 
