@@ -63,13 +63,16 @@ Top1Layout top1_layout(const Geom& g)
     return L;
 }
 
-struct ExactLayout { size_t partial_off, total; DirectPlan dp; };
+struct ExactLayout { size_t partial_off, total; DirectPlan dp; TcPlan tp; bool tc_ok; };
 ExactLayout exact_layout(const Geom& g)
 {
     ExactLayout L;
     L.dp = plan_direct(g);
+    L.tc_ok = plan_tc(g, &L.tp);
     L.partial_off = kWsDataOffset;
-    L.total = align_up(L.partial_off + L.dp.partial_bytes, 256);
+    size_t partial = L.dp.partial_bytes;
+    if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
+    L.total = align_up(L.partial_off + partial, 256);
     return L;
 }
 
@@ -149,11 +152,18 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
-    if (desc->algo == GACONV_ALGO_TENSOR || desc->math == GACONV_MATH_TF32) return GACONV_ERR_UNSUPPORTED;
+    if (desc->math == GACONV_MATH_TF32) return GACONV_ERR_UNSUPPORTED;
     const ExactLayout L = exact_layout(g);
+    if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
     st = check_ws(desc, L.total);
     if (st != GACONV_OK) return st;
     char* ws = static_cast<char*>(desc->workspace);
+    if (L.tc_ok && desc->algo != GACONV_ALGO_DIRECT) {
+        cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
+                                  reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws),
+                                  L.tp, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    }
     cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
                                   reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.dp,
                                   static_cast<cudaStream_t>(stream));

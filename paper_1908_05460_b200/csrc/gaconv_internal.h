@@ -63,4 +63,13 @@ DirectPlan plan_direct(const Geom& g);
 cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
                           const Geom& g, const DirectPlan& plan, cudaStream_t stream);
 
+// ---- exact filter gradient on tcgen05 tensor cores (bf16, NHWC X, shapes its tiling covers) ----
+struct TcPlan {
+    size_t partial_bytes;
+    alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
+};
+bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel
+cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters, uint32_t* status,
+                      const TcPlan& plan, cudaStream_t stream);
+
 }  // namespace gaconv

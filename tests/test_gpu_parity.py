@@ -236,3 +236,40 @@ def test_full_size_layers(net, li, dtype):
         worst = max(worst, abs(got[k, c, r, s_] - v) / nrm)
     assert worst <= tol(dtype)
     assert np.all(np.isfinite(got))
+
+
+# ---- tensor-core (tcgen05) exact path, forced, on shapes that exercise each of its tilings ----
+TC_SHAPES = [
+    ConvLayer("tc 16->16@32 halo M64 ct16", 8, 16, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("tc 32->32@16 ct32", 6, 32, 16, 16, 32, 3, 3, 1, 1),
+    ConvLayer("tc 64->64@8 whole-image chunks", 16, 64, 8, 8, 64, 3, 3, 1, 1),
+    ConvLayer("tc 64->64@32 ct64", 4, 64, 32, 32, 64, 3, 3, 1, 1),
+    ConvLayer("tc 64->128@16 M128", 8, 64, 16, 16, 128, 3, 3, 1, 1),
+    ConvLayer("tc 128->256@8 many tiles", 8, 128, 8, 8, 256, 3, 3, 1, 1),
+    ConvLayer("tc 16->32 stride2", 6, 16, 32, 32, 32, 3, 3, 2, 1),
+    ConvLayer("tc 32->64 stride2", 5, 32, 16, 16, 64, 3, 3, 2, 1),
+    ConvLayer("tc 4x4 maps", 9, 48, 4, 4, 80, 3, 3, 1, 1),
+    ConvLayer("tc 5x5 c64", 3, 64, 16, 16, 64, 5, 5, 1, 2),
+    ConvLayer("tc ragged channels", 4, 40, 16, 16, 24, 3, 3, 1, 1),
+    ConvLayer("tc k72", 4, 16, 8, 8, 72, 3, 3, 1, 1),
+    ConvLayer("tc 1x1", 4, 32, 16, 16, 48, 1, 1, 1, 0),
+    ConvLayer("tc many splits", 128, 16, 32, 32, 16, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("li", range(len(TC_SHAPES)), ids=[l.name for l in TC_SHAPES])
+def test_tensor_core_exact_matches_oracle_and_direct(li):
+    layer = TC_SHAPES[li]
+    x, dy = _inputs(layer, torch.bfloat16, 200 + li)
+    g = GpuLayer(layer, torch.bfloat16, x, dy, alpha=0.25, algo=B.ALGO_TENSOR)
+    got = g.exact()
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+    if layer.n * layer.p * layer.q * layer.k * layer.c <= 3e8:
+        ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.25)
+        assert norm_err(got, ref, dn) <= TOL_BF16
+        assert norm_err(got, ref, dn) <= 1e-4        # bf16 products are exact in fp32: far inside the class tolerance
+    gd = GpuLayer(layer, torch.bfloat16, x, dy, alpha=0.25, algo=B.ALGO_DIRECT)
+    direct = gd.exact()
+    scale = np.maximum(np.abs(direct), 1e-3 * np.abs(direct).max())
+    assert np.max(np.abs(got - direct) / scale) < 1e-2
+    np.testing.assert_array_equal(got, g.exact())                      # reproducible bit for bit
