@@ -157,7 +157,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4], help="layer set: 2 ResNet-20, 3 two-layer CNN, 4 VGG-19")
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
-    ap.add_argument("--layer-iters", type=int, default=10, help="cold per-layer timing iterations")
+    ap.add_argument("--layer-iters", type=int, default=5, help="per-layer timing repetitions (median)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -270,11 +270,15 @@ def main():
     passes = len(slots)
     value = ms_step * 1e3 / (passes * world)
 
-    # ---- per-layer cold timing (L2 flushed before every launch), on the launching stream ----
+    # ---- per-layer timing on the launching stream ----
+    # streamed: a CUDA graph of back-to-back launches of one layer, each on its own copy of the inputs,
+    #   enough copies that a buffer is touched again only after > 2.5x the L2 capacity has streamed by
+    #   (cold data, launch latency amortised as inside the step);
+    # isolated: one launch after a 256 MB L2-flushing write, event to event (includes launch latency).
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def cold_us(fn, iters):
+    def isolated_us(fn, iters):
         ts = []
         for _ in range(iters):
             flush.fill_(1)
@@ -283,12 +287,41 @@ def main():
             ts.append(es.elapsed_time(ee) * 1e3)
         return statistics.median(ts)
 
-    empty_pair_us = cold_us(lambda: None, 20)
+    def streamed_us(s, m, iters):
+        nbytes = (s.x.numel() + s.dy.numel()) * s.eb
+        copies = 48 if m in (B.METHOD_ZERO, B.METHOD_RANDOM) else max(2, min(400, -(-330_000_000 // nbytes)))
+        if m in (B.METHOD_ZERO, B.METHOD_RANDOM):
+            bufs = [(s.x, s.dy)] * copies
+        else:
+            bufs = [(s.x, s.dy)] + [(s.x.clone(), s.dy.clone()) for _ in range(copies - 1)]
+        step_no = 4 * 2 + (3 if m >= 0 else 0)
+
+        def burst():
+            for xb, dyb in bufs:
+                scheds[m].run_layer(s.li, step_no, xb, dyb, s.dw, s.desc)
+        burst()
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            burst()
+        gr.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(iters):
+            es.record(); gr.replay(); ee.record()
+            ee.synchronize()
+            ts.append(es.elapsed_time(ee) * 1e3 / copies)
+        del gr, bufs
+        return statistics.median(ts)
+
+    empty_pair_us = isolated_us(lambda: None, 20)
     table = []
     for s in slots:
         row = {"layer": s.layer.name, "index": s.li, "dtype": s.dname}
         for name, m in methods:
-            row[name + "_us"] = cold_us(lambda: run_one(s, m, 2), args.layer_iters)
+            row[name + "_us"] = streamed_us(s, m, args.layer_iters)
+        for name, m in methods[:2]:
+            row[name + "_isolated_us"] = isolated_us(lambda: run_one(s, m, 2), 5)
         l = s.layer
         fl, be, bt = l.flops_exact(), l.bytes_exact(s.eb), l.bytes_top1(s.eb)
         t_tensor = fl / (peaks["bf16_tflops"] * 1e12 * (1.0 if s.eb == 2 else 0.5)) * 1e6   # tf32 nominal ratio 1/2
@@ -368,10 +401,10 @@ def main():
                                % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), L, ",".join(dtype_names)),
                    "layer_passes_per_step": passes, "cuda_graph": graph is not None,
                    "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
-                         "order); per-layer timings flush L2 with a 256 MB write before every launch" % (input_bytes / 1e6)},
+                         "order); per-layer timings stream over rotating input copies > 2.5x L2" % (input_bytes / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
-        "breakdown_us": {"cold_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
+        "breakdown_us": {"streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
                          "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
                          "top1_speedup_over_exact": sum_us["exact"] / sum_us["top1"]},
         "paper_context": "paper reports >7% training wall-clock speedup (ResNet-20/VGG-19, Titan Xp, TF 1.13, cuDNN 7.4.2)",

@@ -1,13 +1,18 @@
 // Exact filter gradient on the FP32 pipes (paper Section 2.4: "to compute df we have to convolve I
 // with dO"):   dW[k,c,r,s] = alpha * sum_{n,p,q} Xz[n,c,p*st+r-pad,q*st+s-pad] * dY[n,k,p,q].
 // Works for every shape, layout and dtype: products and sums are fp32, so fp32 inputs meet the
-// fp32 tolerance class.  It is the anchor the tensor-core path is checked against on shapes the
-// oracle cannot cover in full, and the route for shapes the tensor-core path does not tile.
+// fp32 tolerance class.  It serves fp32 inputs, the 3-channel stem layers and every shape the
+// tensor-core path does not tile.
 //
-// Tiled kernel: a CTA owns a 16 (k) x 16 (c) x R x S block of dW and a range of work items; a work
-// item is one image's band of BP x BQ output pixels.  Per item the dY band and the X window are
-// staged in shared memory as fp32; thread (tk, tc) keeps its R*S accumulators in registers.
-// Splits of the reduction are combined by the last CTA to finish, in split order.
+// Register-tiled kernel.  A CTA owns a (TKT*OTK) x (TCT*OTC) block of (k, c) with all R*S filter
+// taps, and a contiguous range of work items; an item is one image's band of BP x BQ output pixels.
+// Per item the dY band is staged in shared memory pixel-major ([k-group][pixel][TKT]) and the X
+// window channel-minor ([row][col][c]), both as fp32.  The OTK*OTC "output threads" of a pixel
+// group each keep TKT*TCT*R*S accumulators in registers; the 128/(OTK*OTC) pixel groups take the
+// band's pixels round-robin, so one vector load of dY and R*S vector loads of X feed
+// TKT*TCT*R*S FMAs.  At the end the pixel groups are summed (warp shuffles, then shared memory, in a
+// fixed order) and the CTA writes its block: to dW if it is the only split, else to its slot of
+// the partial buffer, which reduce_splits() adds up in split order.
 #include "gaconv_internal.h"
 
 namespace gaconv {
@@ -19,26 +24,34 @@ template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloa
     return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
 }
 
-constexpr int TK = 16, TC = 16;
+constexpr int kThreads = 128;
 
-template <typename T, int R, int S>
-__global__ void __launch_bounds__(256)
+template <int N> struct Vec;
+template <> struct Vec<1> { float v[1]; __device__ void load(const float* p) { v[0] = *p; } };
+template <> struct Vec<2> { float v[2]; __device__ void load(const float* p) { float2 t = *reinterpret_cast<const float2*>(p); v[0] = t.x; v[1] = t.y; } };
+template <> struct Vec<4> { float v[4]; __device__ void load(const float* p) { float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; } };
+
+template <typename T, int R, int S, int TKT, int TCT, int OTK, int OTC>
+__global__ void __launch_bounds__(kThreads)
 direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw,
-                    float* __restrict__ partial, uint32_t* __restrict__ counters, Geom g, DirectPlan pl)
+                    float* __restrict__ partial, Geom g, DirectPlan pl)
 {
-    extern __shared__ float smem[];
+    constexpr int TK = TKT * OTK, TC = TCT * OTC, OT = OTK * OTC, PG = kThreads / OT, ACC = TKT * TCT * R * S;
+    static_assert(kThreads % OT == 0 && OT <= 64, "output threads must divide the CTA");
+    extern __shared__ __align__(16) float smem[];
+    const int npx = pl.bp * pl.bq;
     const int win_h = (pl.bp - 1) * g.stride_h + R, win_w = (pl.bq - 1) * g.stride_w + S;
-    float* s_dy = smem;                                  // [TK][bp*bq]
-    float* s_x = smem + TK * pl.bp * pl.bq;              // [win_h][win_w][TC]
-    __shared__ bool s_last;
+    float* s_dy = smem;                          // [OTK][npx][TKT]
+    float* s_x = smem + TK * npx;                // [win_h][win_w][TC]
 
     const int tile = blockIdx.x, split = blockIdx.y;
     const int k0 = (tile / pl.tiles_c) * TK, c0 = (tile % pl.tiles_c) * TC;
-    const int tk = threadIdx.x / TC, tc = threadIdx.x % TC;
+    const int ot = threadIdx.x % OT, pg = threadIdx.x / OT;
+    const int otk = ot / OTC, otc = ot % OTC;
 
-    float acc[R * S];
+    float acc[ACC];
 #pragma unroll
-    for (int i = 0; i < R * S; ++i) acc[i] = 0.f;
+    for (int i = 0; i < ACC; ++i) acc[i] = 0.f;
 
     const int per = (pl.items + pl.splits - 1) / pl.splits;
     const int it_end = min(pl.items, (split + 1) * per);
@@ -47,15 +60,16 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
         const int band = it % (pl.bands_p * pl.bands_q);
         const int p0 = (band / pl.bands_q) * pl.bp, q0 = (band % pl.bands_q) * pl.bq;
         __syncthreads();
-        for (int i = threadIdx.x; i < TK * pl.bp * pl.bq; i += blockDim.x) {
-            const int kk = i / (pl.bp * pl.bq), j = i % (pl.bp * pl.bq);
+        // dY band: coalesced along pixels, stored as [k-group][pixel][TKT]
+        for (int i = threadIdx.x; i < TK * npx; i += kThreads) {
+            const int kk = i / npx, j = i % npx;
             const int p = p0 + j / pl.bq, q = q0 + j % pl.bq, k = k0 + kk;
             float v = 0.f;
             if (k < g.k && p < g.p && q < g.q) v = ldf(dy + (((long long)n * g.k + k) * g.p + p) * g.q + q);
-            s_dy[i] = v;
+            s_dy[((kk / TKT) * npx + j) * TKT + kk % TKT] = v;
         }
         const int h0 = p0 * g.stride_h - g.pad_h, w0 = q0 * g.stride_w - g.pad_w;
-        for (int i = threadIdx.x; i < win_h * win_w * TC; i += blockDim.x) {
+        for (int i = threadIdx.x; i < win_h * win_w * TC; i += kThreads) {
             const int cc = i % TC, pix = i / TC;
             const int hh = h0 + pix / win_w, ww = w0 + pix % win_w, c = c0 + cc;
             float v = 0.f;
@@ -64,44 +78,63 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
             s_x[i] = v;
         }
         __syncthreads();
-        for (int pp = 0; pp < pl.bp; ++pp)
-            for (int qq = 0; qq < pl.bq; ++qq) {
-                const float d = s_dy[(tk * pl.bp + pp) * pl.bq + qq];
-                const float* xb = s_x + ((pp * g.stride_h) * win_w + qq * g.stride_w) * TC + tc;
+        for (int j = pg; j < npx; j += PG) {
+            const int pp = j / pl.bq, qq = j % pl.bq;
+            Vec<TKT> d;
+            d.load(s_dy + (otk * npx + j) * TKT);
+            const float* xb = s_x + ((pp * g.stride_h) * win_w + qq * g.stride_w) * TC + otc * TCT;
 #pragma unroll
-                for (int r = 0; r < R; ++r)
+            for (int r = 0; r < R; ++r)
 #pragma unroll
-                    for (int s = 0; s < S; ++s) acc[r * S + s] = fmaf(d, xb[(r * win_w + s) * TC], acc[r * S + s]);
-            }
+                for (int s = 0; s < S; ++s) {
+                    Vec<TCT> xv;
+                    xv.load(xb + (r * win_w + s) * TC);
+#pragma unroll
+                    for (int a = 0; a < TKT; ++a)
+#pragma unroll
+                        for (int b = 0; b < TCT; ++b)
+                            acc[((a * TCT + b) * R + r) * S + s] = fmaf(d.v[a], xv.v[b], acc[((a * TCT + b) * R + r) * S + s]);
+                }
+        }
     }
 
-    const int k = k0 + tk, c = c0 + tc;
-    const bool valid = k < g.k && c < g.c;
-    if (pl.splits == 1) {
-        if (valid)
+    // ---- sum the pixel groups: lanes first (groups that share a warp), then warps through shared memory ----
+    constexpr int kWarps = kThreads / 32;
 #pragma unroll
-            for (int i = 0; i < R * S; ++i) dw[k * g.ws_k + c * g.ws_c + (i / S) * g.ws_r + (i % S) * g.ws_s] = g.alpha * acc[i];
-        return;
-    }
-    // partial[split][tile][rs][thread]
-    const size_t tile_elems = (size_t)R * S * 256;
-    float* mine = partial + ((size_t)split * gridDim.x + tile) * tile_elems;
+    for (int off = OT; off < 32; off <<= 1)
 #pragma unroll
-    for (int i = 0; i < R * S; ++i) mine[i * 256 + threadIdx.x] = acc[i];
-    __threadfence();
+        for (int i = 0; i < ACC; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], off);
+    // what is left per output thread: one partial sum per warp (OT < 32) or per pixel group (OT >= 32)
+    constexpr int SETS = OT >= 32 ? PG : kWarps;
+    constexpr int CH = 16;                                           // accumulators exchanged per pass
     __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&counters[tile % kWsNumCounters], 1u) == (uint32_t)pl.splits - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
+    float* s_red = smem;                                             // [SETS][OT][CH]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool owner = OT >= 32 ? true : lane < OT;
+    const int set = OT >= 32 ? pg : warp;
+    float* out = pl.splits == 1 ? dw : partial + (size_t)split * g.k * g.c * R * S;
+    const float scale = pl.splits == 1 ? g.alpha : 1.0f;
 #pragma unroll
-    for (int i = 0; i < R * S; ++i) {
-        float tot = 0.f;
-        for (int sp = 0; sp < pl.splits; ++sp)
-            tot += __ldcg(partial + ((size_t)sp * gridDim.x + tile) * tile_elems + i * 256 + threadIdx.x);
-        if (valid) dw[k * g.ws_k + c * g.ws_c + (i / S) * g.ws_r + (i % S) * g.ws_s] = g.alpha * tot;
+    for (int base = 0; base < ACC; base += CH) {
+        if (owner) {
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+                if (base + i < ACC) s_red[(set * OT + ot) * CH + i] = acc[base + i];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < OT * CH; e += kThreads) {
+            const int o = e / CH, i = e % CH, ai = base + i;
+            if (ai < ACC) {
+                float tot = 0.f;
+#pragma unroll
+                for (int w = 0; w < SETS; ++w) tot += s_red[(w * OT + o) * CH + i];
+                const int a = ai / (TCT * R * S), b = (ai / (R * S)) % TCT, r = (ai / S) % R, s = ai % S;
+                const int k = k0 + (o / OTC) * TKT + a, c = c0 + (o % OTC) * TCT + b;
+                if (k < g.k && c < g.c) out[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = scale * tot;
+            }
+        }
+        __syncthreads();
     }
-    if (threadIdx.x == 0) counters[tile % kWsNumCounters] = 0;
 }
 
 // Any filter size: one thread per dW element, whole reduction in the thread.
@@ -130,9 +163,27 @@ direct_element_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* 
     dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * acc;
 }
 
+// thread-tile shape of each variant
+struct Variant { int tkt, tct, otk, otc; };
+Variant variant_for(const Geom& g)
+{
+    const bool narrow = g.c <= 4;
+    if (g.r == 5) return narrow ? Variant{1, 4, 16, 1} : Variant{2, 2, 8, 8};
+    return narrow ? Variant{4, 4, 4, 1} : Variant{4, 4, 4, 4};
+}
+
+size_t smem_for(const Geom& g, const Variant& v, int bp, int bq)
+{
+    const int tk = v.tkt * v.otk, tc = v.tct * v.otc, ot = v.otk * v.otc;
+    const size_t stage = sizeof(float) * ((size_t)tk * bp * bq + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * tc);
+    const int sets = ot >= 32 ? kThreads / ot : kThreads / 32;
+    const size_t red = sizeof(float) * (size_t)sets * ot * 16;
+    return stage > red ? stage : red;
+}
+
 template <typename T>
-cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_t* counters, const Geom& g,
-                     const DirectPlan& pl, cudaStream_t stream)
+cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, const Geom& g, const DirectPlan& pl,
+                     cudaStream_t stream)
 {
     if (!pl.tiled) {
         const long long total = (long long)g.k * g.r * g.s * g.c;
@@ -140,20 +191,28 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_
         note_launch();
         return cudaGetLastError();
     }
-    const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
-    const size_t smem = sizeof(float) * ((size_t)TK * pl.bp * pl.bq + (size_t)win_h * win_w * TC);
+    const Variant v = variant_for(g);
+    const size_t smem = smem_for(g, v, pl.bp, pl.bq);
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
-#define GACONV_DIRECT_CASE(RR, SS)                                                                         \
-    if (g.r == RR && g.s == SS) {                                                                          \
-        direct_tiled_kernel<T, RR, SS><<<grid, 256, smem, stream>>>(x, dy, dw, partial, counters, g, pl); \
-        note_launch();                                                                                     \
-        return cudaGetLastError();                                                                         \
+    bool done = false;
+#define GACONV_DIRECT_CASE(RR, A, B, C, D)                                                                     \
+    if (!done && g.r == RR && v.tkt == A && v.tct == B && v.otk == C && v.otc == D) {                          \
+        direct_tiled_kernel<T, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
+        done = true;                                                                                           \
     }
-    GACONV_DIRECT_CASE(1, 1)
-    GACONV_DIRECT_CASE(3, 3)
-    GACONV_DIRECT_CASE(5, 5)
+    GACONV_DIRECT_CASE(1, 4, 4, 4, 4)
+    GACONV_DIRECT_CASE(1, 4, 4, 4, 1)
+    GACONV_DIRECT_CASE(3, 4, 4, 4, 4)
+    GACONV_DIRECT_CASE(3, 4, 4, 4, 1)
+    GACONV_DIRECT_CASE(5, 2, 2, 8, 8)
+    GACONV_DIRECT_CASE(5, 1, 4, 16, 1)
 #undef GACONV_DIRECT_CASE
-    return cudaErrorInvalidValue;
+    if (!done) return cudaErrorInvalidValue;
+    note_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (pl.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.c * g.r * g.s, pl.splits, g.alpha, stream);
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -162,40 +221,41 @@ DirectPlan plan_direct(const Geom& g)
 {
     DirectPlan pl{};
     pl.tiled = (g.r == g.s) && (g.r == 1 || g.r == 3 || g.r == 5);
-    pl.tiles_k = (g.k + TK - 1) / TK;
-    pl.tiles_c = (g.c + TC - 1) / TC;
+    const Variant v = variant_for(g);
+    const int tk = v.tkt * v.otk, tc = v.tct * v.otc;
+    pl.tiles_k = (g.k + tk - 1) / tk;
+    pl.tiles_c = (g.c + tc - 1) / tc;
     pl.bq = g.q < 32 ? g.q : 32;
-    pl.bp = g.p < 4 ? g.p : 4;
-    while (pl.bp * 2 <= g.p && pl.bp * pl.bq < 128) pl.bp *= 2;
-    // shared memory must stay under the default 48 KiB
-    auto smem = [&](int bp, int bq) {
-        return sizeof(float) * ((size_t)TK * bp * bq + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * TC);
-    };
-    while (pl.bp > 1 && smem(pl.bp, pl.bq) > 40 * 1024) pl.bp /= 2;
-    while (pl.bq > 1 && smem(pl.bp, pl.bq) > 40 * 1024) pl.bq /= 2;
+    pl.bp = 1;
+    while (pl.bp * 2 <= g.p && pl.bp * 2 * pl.bq <= 256 && smem_for(g, v, pl.bp * 2, pl.bq) <= 44 * 1024) pl.bp *= 2;
+    while (pl.bq > 1 && smem_for(g, v, pl.bp, pl.bq) > 44 * 1024) pl.bq /= 2;
     pl.bands_p = (g.p + pl.bp - 1) / pl.bp;
     pl.bands_q = (g.q + pl.bq - 1) / pl.bq;
     pl.items = g.n * pl.bands_p * pl.bands_q;
     const int tiles = pl.tiles_k * pl.tiles_c;
-    int splits = (148 * 4 + tiles - 1) / tiles;
+    // about three CTAs per SM; each split's partial block is written once and read once
+    int splits = (148 * 3 + tiles - 1) / tiles;
     if (splits > pl.items) splits = pl.items;
-    if (tiles > kWsNumCounters) splits = 1;
-    const size_t tile_bytes = (size_t)g.r * g.s * 256 * sizeof(float);
-    while (splits > 1 && (size_t)splits * tiles * tile_bytes > ((size_t)64 << 20)) --splits;
+    const size_t out_bytes = (size_t)g.k * g.c * g.r * g.s * sizeof(float);
+    while (splits > 1 && (size_t)splits * out_bytes > ((size_t)96 << 20)) --splits;
     if (splits < 1) splits = 1;
+    {   // no empty splits
+        const int per = (pl.items + splits - 1) / splits;
+        splits = (pl.items + per - 1) / per;
+    }
     if (!pl.tiled) splits = 1;
     pl.splits = splits;
-    pl.partial_bytes = splits > 1 ? (size_t)splits * tiles * tile_bytes : 0;
+    pl.partial_bytes = splits > 1 ? (size_t)splits * out_bytes : 0;
     return pl;
 }
 
 cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
                           const Geom& g, const DirectPlan& plan, cudaStream_t stream)
 {
+    (void)counters;
     if (g.bf16)
-        return launch_t(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy), dw, partial,
-                        counters, g, plan, stream);
-    return launch_t(static_cast<const float*>(x), static_cast<const float*>(dy), dw, partial, counters, g, plan, stream);
+        return launch_t(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy), dw, partial, g, plan, stream);
+    return launch_t(static_cast<const float*>(x), static_cast<const float*>(dy), dw, partial, g, plan, stream);
 }
 
 }  // namespace gaconv

@@ -31,6 +31,9 @@ struct Geom {
     float alpha;
 };
 
+// ---- fixed-order sum of split partials: dw = alpha * sum_sp partial[sp][0..count) ----
+cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int splits, float alpha, cudaStream_t stream);
+
 // ---- selection (Algorithm 1, arg-max and sum lines) ----
 cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_sparse, const Geom& g,
                           cudaStream_t stream);

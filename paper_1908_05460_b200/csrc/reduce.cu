@@ -1,0 +1,59 @@
+// Fixed-order sum of split partial results:  dw[i] = alpha * sum_{sp} partial[sp][i], i < count.
+// partial is [splits][count] in the element order of dw.  A block handles 32 columns (float4 columns
+// when count is a multiple of four); each of its 32 warps sums an interleaved subset of the splits in
+// ascending order, and warp 0 adds the 32 subtotals in warp order, so the result does not depend
+// on scheduling.
+#include "gaconv_internal.h"
+
+namespace gaconv {
+namespace {
+
+constexpr int kReduceWarps = 32;
+
+template <typename V> __device__ __forceinline__ V vzero();
+template <> __device__ __forceinline__ float vzero<float>() { return 0.f; }
+template <> __device__ __forceinline__ float4 vzero<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ void vadd(float& a, const float b) { a += b; }
+__device__ __forceinline__ void vadd(float4& a, const float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+__device__ __forceinline__ float vscale(float a, float s) { return a * s; }
+__device__ __forceinline__ float4 vscale(float4 a, float s) { return make_float4(a.x * s, a.y * s, a.z * s, a.w * s); }
+
+template <typename V>
+__global__ void __launch_bounds__(32 * kReduceWarps)
+reduce_splits_kernel(const V* __restrict__ partial, V* __restrict__ dw, size_t count, int splits, float alpha)
+{
+    __shared__ V sm[kReduceWarps][32];
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const size_t i = (size_t)blockIdx.x * 32 + lane;
+    V acc = vzero<V>();
+    if (i < count) {
+        const V* p = partial + i;
+#pragma unroll 5
+        for (int sp = grp; sp < splits; sp += kReduceWarps) vadd(acc, __ldcg(p + (size_t)sp * count));
+    }
+    sm[grp][lane] = acc;
+    __syncthreads();
+    if (grp == 0 && i < count) {
+        V t = sm[0][lane];
+        const int used = splits < kReduceWarps ? splits : kReduceWarps;
+        for (int w = 1; w < used; ++w) vadd(t, sm[w][lane]);
+        dw[i] = vscale(t, alpha);
+    }
+}
+
+}  // namespace
+
+cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int splits, float alpha, cudaStream_t stream)
+{
+    if (count % 4 == 0) {
+        const size_t c4 = count / 4;
+        reduce_splits_kernel<float4><<<(unsigned)((c4 + 31) / 32), 32 * kReduceWarps, 0, stream>>>(
+            reinterpret_cast<const float4*>(partial), reinterpret_cast<float4*>(dw), c4, splits, alpha);
+    } else {
+        reduce_splits_kernel<float><<<(unsigned)((count + 31) / 32), 32 * kReduceWarps, 0, stream>>>(partial, dw, count, splits, alpha);
+    }
+    note_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace gaconv

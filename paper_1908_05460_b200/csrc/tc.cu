@@ -14,7 +14,7 @@
 //   D  = R accumulators in tensor memory, fp32.  With M = 64 (K <= 64) an accumulator occupies 16 of
 //        the 32 lanes of each TMEM sub-partition, so two accumulators share the same columns.
 // A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks; the
-// partial blocks of the splits are combined by the last CTA to finish, in split order.
+// partial blocks of the splits are summed in split order by a second, element-parallel kernel.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue.
 // Every mbarrier wait is bounded; on expiry the kernel raises the workspace status word, drains
@@ -51,6 +51,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// Same bound in wall time, but the warp sleeps between polls so that it does not take issue slots
+// from the producer and MMA threads while the main loop runs.
+__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(128);
+    }
+    return false;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
@@ -63,36 +72,20 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
+// Issues the load only; the caller executes tcgen05.wait::ld before reading v.
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float (&v)[16]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]),
+                   "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15])
                  : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor: start address, leading/stride byte offsets (16-byte units),
-// descriptor version 1, swizzle code in bits 61..63 (2 = 128 B, 4 = 64 B, 6 = 32 B).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t swz_code) {
-    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo >> 4) & 0x3fffu) << 16) |
-           ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46) | ((uint64_t)swz_code << 61);
-}
-
 struct TcParams {
     Geom g;
     int m;              // MMA M: 64 or 128 output channels per k-tile
@@ -114,10 +107,14 @@ struct TcParams {
     int ksteps;         // ci*bp*Q/16
     int tmem_cols;      // power of two >= 32
     uint32_t idesc;
+    int timeline;       // 1: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
 };
 
 constexpr int kMaxStages = 8;
 
+// R_T: filter rows (0 = take it from the geometry); KS_T: k-steps per A box (0 = from the plan).
+// The compile-time values let the issue loop unroll into straight-line MMA instructions.
+template <int R_T, int KS_T>
 __global__ void __launch_bounds__(192, 1)
 exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
                 float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters,
@@ -127,7 +124,6 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ bool s_last;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -154,90 +150,153 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = s_tmem_base;
+    long long* tl = (P.timeline && blockIdx.x == 0 && blockIdx.y == 0) ? reinterpret_cast<long long*>(status + 16) : nullptr;
+    if (tl && threadIdx.x == 0) tl[0] = clock64();
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
-        int issued = 0;
+        // chunk coordinates advance incrementally: no division inside the loop
+        int n0, p0;
+        const bool whole_maps = P.a_sub_px < 64;
+        const int cpi = whole_maps ? 1 : g.p / P.bp;
+        if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
+        else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
+        const uint32_t tx_bytes = P.a_subs * P.a_sub_bytes + P.b_tiles * P.b_tile_bytes;
+        int issued = 0, st = 0, ph = 0;
         for (int it = 0; it < nchunks; ++it) {
-            const int st = it % P.stages;
-            if (it >= P.stages && !mbar_wait(smem_u32(&bar_empty[st]), ((it / P.stages) - 1) & 1)) { s_abort = 1; atomicOr(status, 1u); break; }
+            if (it >= P.stages && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1)) { s_abort = 1; atomicOr(status, 1u); break; }
             if (s_abort) break;
-            const int ch = ch_begin + it;
             const uint32_t full = smem_u32(&bar_full[st]);
             const uint32_t sa = smem_base + st * P.stage_bytes;
-            const uint32_t sb = sa + P.a_region_bytes;
-            mbar_expect_tx(full, P.a_subs * P.a_sub_bytes + P.b_tiles * P.b_tile_bytes);
-            int n0, p0;
-            if (P.ci > 1 || P.a_sub_px < 64) { n0 = ch * P.ci; p0 = 0; }
-            else { const int cpi = g.p / P.bp; n0 = ch / cpi; p0 = (ch % cpi) * P.bp; }
-            if (P.a_sub_px < 64) {
+            uint32_t sb = sa + P.a_region_bytes;
+            mbar_expect_tx(full, tx_bytes);
+            if (whole_maps) {
                 tma_load_3d(sa, &map_dy, full, 0, k0, n0);                       // ci whole maps in one box
             } else {
-                for (int b = 0; b < P.a_subs; ++b) tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, p0 * g.q + 64 * b, k0, n0);
+                int px = p0 * g.q;
+                for (int b = 0; b < P.a_subs; ++b, px += 64) tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, px, k0, n0);
             }
-            for (int t = 0; t < P.b_tiles; ++t) {
-                const int s = t % g.s, r = t / g.s;
-                const int h0 = P.halo ? p0 - g.pad_h : p0 * g.stride_h + r - g.pad_h;
-                tma_load_4d(sb + t * P.b_tile_stride, &map_x, full, c0, s - g.pad_w, h0, n0);
+            if (P.halo) {
+                for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride) tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 - g.pad_h, n0);
+            } else {
+                for (int r = 0; r < g.r; ++r)
+                    for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride)
+                        tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 * g.stride_h + r - g.pad_h, n0);
             }
             ++issued;
+            if (whole_maps) n0 += P.ci;
+            else { p0 += P.bp; if (p0 >= g.p) { p0 = 0; ++n0; } }
+            if (++st == P.stages) { st = 0; ph ^= 1; }
         }
         if (s_abort) {   // drain: wait (bounded) for the copies already issued
             for (int it = max(0, issued - P.stages); it < issued; ++it) mbar_wait(smem_u32(&bar_full[it % P.stages]), (it / P.stages) & 1);
         }
     } else if (warp == 1 && lane == 0) {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t a_row_bytes = P.a_sub_px * 2, a_sbo = 8 * a_row_bytes;
-        const uint32_t b_row_bytes = P.ct * 2, b_sbo = 8 * b_row_bytes;
+        // descriptors are assembled from a constant high word and a low word that only advances
+        const uint32_t a_row_bytes = P.a_sub_px * 2, b_row_bytes = P.ct * 2;
+        const uint32_t a_hi = ((8 * a_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.a_swz << 29);
+        const uint32_t b_hi = ((8 * b_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
+        const uint32_t a_lo_c = 1u << 16, b_lo_c = (((uint32_t)P.b_tile_stride >> 4) & 0x3fffu) << 16;
         const int ks_per_sub = P.a_sub_px / 16;
-        bool ok = true;
-        for (int it = 0; it < nchunks && ok; ++it) {
-            const int st = it % P.stages;
-            if (!mbar_wait(smem_u32(&bar_full[st]), (it / P.stages) & 1)) { s_abort = 1; atomicOr(status, 1u); ok = false; break; }
+        const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4, b_k_step = (16 * b_row_bytes) >> 4;
+        const uint32_t b_r_step = (P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
+        const uint32_t d_step_even = P.m == 128 ? (uint32_t)nmma : (16u << 16);                 // r -> r+1, r even
+        const uint32_t d_step_odd = P.m == 128 ? (uint32_t)nmma : (uint32_t)nmma - (16u << 16);  // r -> r+1, r odd
+        const int R = R_T ? R_T : g.r;
+        const int KS = KS_T ? KS_T : ks_per_sub;
+        const uint64_t a_hi64 = (uint64_t)a_hi << 32, b_hi64 = (uint64_t)b_hi << 32;
+        const uint32_t idesc = P.idesc;
+        int st = 0, ph = 0;
+        bool fresh = true;            // the next k-step starts the accumulation (overwrites TMEM)
+        for (int it = 0; it < nchunks; ++it) {
+            if (!mbar_wait(smem_u32(&bar_full[st]), ph)) { s_abort = 1; atomicOr(status, 1u); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (tl && it == 0) tl[1] = clock64();
             const uint32_t sa = smem_base + st * P.stage_bytes;
-            const uint32_t sb = sa + P.a_region_bytes;
-            for (int kk = 0; kk < P.ksteps; ++kk) {
-                const uint64_t adesc = smem_desc(sa + (kk / ks_per_sub) * P.a_sub_bytes + (kk % ks_per_sub) * 32, 16, a_sbo, P.a_swz);
-                for (int r = 0; r < g.r; ++r) {
-                    const uint32_t baddr = sb + (P.halo ? 0 : r * g.s * P.b_tile_stride) + (16 * kk + (P.halo ? r * g.q : 0)) * b_row_bytes;
-                    const uint64_t bdesc = smem_desc(baddr, P.b_tile_stride, b_sbo, P.b_swz);
-                    const uint32_t d = P.m == 128 ? tmem_base + r * nmma : tmem_base + (((uint32_t)(r & 1) * 16u) << 16) + (r >> 1) * nmma;
-                    umma_bf16(d, adesc, bdesc, P.idesc, (it > 0 || kk > 0) ? 1u : 0u);
+            uint32_t a_lo = a_lo_c | (sa >> 4);
+            uint32_t b_lo = b_lo_c | ((sa + P.a_region_bytes) >> 4);
+            for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
+                if (fresh) {      // first k-step of this CTA: accumulate flag off
+                    uint32_t d = tmem_base, bl = b_lo;
+#pragma unroll
+                    for (int r = 0; r < R; ++r, bl += b_r_step) {
+                        umma_bf16(d, a_hi64 | a_lo, b_hi64 | bl, idesc, 0u);
+                        d += (r & 1) ? d_step_odd : d_step_even;
+                    }
                 }
+#pragma unroll
+                for (int k4 = 0; k4 < KS; ++k4) {
+                    if (!(fresh && k4 == 0)) {
+                        uint32_t d = tmem_base, bl = b_lo + k4 * b_k_step;
+#pragma unroll
+                        for (int r = 0; r < R; ++r, bl += b_r_step) {
+                            umma_bf16_acc(d, a_hi64 | (a_lo + 2 * k4), b_hi64 | bl, idesc);
+                            d += (r & 1) ? d_step_odd : d_step_even;
+                        }
+                    }
+                }
+                fresh = false;
+                b_lo += KS * b_k_step;
             }
             umma_commit(smem_u32(&bar_empty[st]));   // frees the stage once these MMAs have read it
+            if (++st == P.stages) { st = 0; ph ^= 1; }
         }
         umma_commit(smem_u32(&bar_acc));             // accumulators complete
+        if (tl) tl[2] = clock64();
     } else if (warp >= 2) {
         // ------------------------------------------------------------------ epilogue: TMEM -> global
-        const bool ready = mbar_wait(smem_u32(&bar_acc), 0);
+        const bool ready = mbar_wait_sleepy(smem_u32(&bar_acc), 0);
         if (!ready) { s_abort = 1; atomicOr(status, 1u); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (tl && threadIdx.x == 64) tl[3] = clock64();
         if (ready && !s_abort) {
             const int sp = warp & 3;
             float* out = P.splits == 1 ? dw : partial + (size_t)split * g.k * g.r * g.s * g.c;
-            const float scale = P.splits == 1 ? g.alpha : 1.0f;
+            const float scale = nchunks > 0 ? (P.splits == 1 ? g.alpha : 1.0f) : 0.0f;
             const int groups = P.m == 128 ? g.r : (g.r + 1) / 2;
+            const int k = k0 + (P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15));
+            const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
             for (int gi = 0; gi < groups; ++gi) {
                 const int r = P.m == 128 ? gi : 2 * gi + (lane >> 4);
-                const int k = k0 + (P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15));
-                const bool row_ok = r < g.r && k < g.k && (nchunks > 0 || true);
-                for (int j0 = 0; j0 < nmma; j0 += 16) {
-                    float v[16];
-                    const uint32_t taddr = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma + j0;
-                    if (nmma - j0 >= 16) tmem_ld16(taddr, v); else tmem_ld8(taddr, v);
-                    if (!row_ok) continue;
-                    const int lim = min(16, nmma - j0);
-                    for (int jj = 0; jj < lim; ++jj) {
-                        const int nn = j0 + jj, s = nn / P.ct, c = c0 + nn % P.ct;
-                        if (c < g.c) out[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = nchunks > 0 ? scale * v[jj] : 0.0f;
+                const bool row_ok = r < g.r && k < g.k;
+                float* row = out + k * g.ws_k + r * g.ws_r;
+                const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
+                for (int s = 0; s < g.s; ++s) {
+                    float* ps = row + s * g.ws_s;
+                    for (int cc = 0; cc < P.ct; cc += 64) {
+                        const uint32_t taddr = tbase + s * P.ct + cc;
+                        // up to four 16-column loads in flight before the single wait
+                        float v[4][16];
+                        const int nld = min(4, (P.ct - cc) >> 4);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (u < nld) tmem_ld16_nowait(taddr + 16 * u, v[u]);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (!row_ok) continue;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (u >= nld) continue;
+                            const int c = c0 + cc + 16 * u;
+                            if (vec && c + 16 <= g.c) {
+                                float4* p4 = reinterpret_cast<float4*>(ps + c);
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4)
+                                    p4[q4] = make_float4(scale * v[u][4 * q4], scale * v[u][4 * q4 + 1],
+                                                         scale * v[u][4 * q4 + 2], scale * v[u][4 * q4 + 3]);
+                            } else {
+#pragma unroll
+                                for (int jj = 0; jj < 16; ++jj)
+                                    if (c + jj < g.c) ps[(c + jj) * g.ws_c] = scale * v[u][jj];
+                            }
+                        }
                     }
                 }
             }
         }
     }
 
+    if (tl && threadIdx.x == 64) tl[4] = clock64();
     // ---------------------------------------------------------------------- teardown
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -245,27 +304,6 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(P.tmem_cols) : "memory");
     }
-    if (P.splits == 1 || s_abort) return;
-
-    // ---------------------------------------------------------------------- split reduction (last CTA of the tile)
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&counters[tile % kWsNumCounters], 1u) == (uint32_t)P.splits - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const int rows = min(P.m, g.k - k0), cols = min(P.ct, g.c - c0);
-    const int per_row = g.r * g.s * cols;
-    const size_t kcrs = (size_t)g.k * g.r * g.s * g.c;
-    for (int e = threadIdx.x; e < rows * per_row; e += blockDim.x) {
-        const int kk = e / per_row, rem = e % per_row;
-        const int r = rem / (g.s * cols), s = (rem / cols) % g.s, c = c0 + rem % cols;
-        const size_t off = (k0 + kk) * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s;
-        float tot = 0.f;
-        for (int sp = 0; sp < P.splits; ++sp) tot += __ldcg(partial + sp * kcrs + off);
-        dw[off] = g.alpha * tot;
-    }
-    if (threadIdx.x == 0) counters[tile % kWsNumCounters] = 0;
 }
 
 // ---------------------------------------------------------------- host side
@@ -377,6 +415,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
         splits = (P.chunks + per - 1) / per;
     }
     P.splits = splits;
+    P.timeline = env_int("GACONV_TC_TIMELINE", 0);
 
     out->partial_bytes = splits > 1 ? (size_t)splits * g.k * g.r * g.s * g.c * 4 : 0;
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
@@ -417,15 +456,30 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     // dynamic shared memory: stages, 1 KiB of alignment slack, and a tail so that the MMA's read of
     // all M rows of an A box with fewer valid rows stays inside the allocation
     const size_t smem = (size_t)P.stages * P.stage_bytes + 1024 + (size_t)P.m * 128;
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(exact_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
     dim3 grid(P.tiles_k * P.tiles_c, P.splits);
-    exact_tc_kernel<<<grid, 192, smem, stream>>>(map_dy, map_x, dw, partial, counters, status, P);
+    const int ks = P.a_sub_px / 16;
+    cudaError_t err = cudaErrorInvalidValue;
+#define GACONV_TC_CASE(RR, KK)                                                                                     \
+    if (err == cudaErrorInvalidValue && (RR == 0 || (g.r == RR && ks == KK))) {                                     \
+        static size_t configured = 0;                                                                              \
+        err = cudaSuccess;                                                                                         \
+        if (smem > configured) {                                                                                   \
+            err = cudaFuncSetAttribute(exact_tc_kernel<RR, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            if (err == cudaSuccess) configured = smem;                                                             \
+        }                                                                                                          \
+        if (err == cudaSuccess)                                                                                    \
+            exact_tc_kernel<RR, KK><<<grid, 192, smem, stream>>>(map_dy, map_x, dw, partial, counters, status, P);  \
+    }
+    GACONV_TC_CASE(3, 4)
+    GACONV_TC_CASE(3, 1)
+    GACONV_TC_CASE(5, 4)
+    GACONV_TC_CASE(1, 4)
+    GACONV_TC_CASE(0, 0)
+#undef GACONV_TC_CASE
+    if (err != cudaSuccess) return err;
     note_launch();
+    if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+    if (P.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.r * g.s * g.c, P.splits, g.alpha, stream);
     return cudaGetLastError();
 }
 
