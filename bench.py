@@ -316,7 +316,7 @@ def main():
 
     empty_pair_us = isolated_us(lambda: None, 20)
     table = []
-    for s in slots:
+    for s in (slots if args.layer_iters > 0 else []):
         row = {"layer": s.layer.name, "index": s.li, "dtype": s.dname}
         for name, m in methods:
             row[name + "_us"] = streamed_us(s, m, args.layer_iters)
@@ -335,9 +335,11 @@ def main():
         table.append(row)
     sum_us = {name: sum(r[name + "_us"] for r in table) for name, _ in methods}
 
-    # ---- roofline of the dominant kernel family (largest share of the cold per-layer time) ----
+    # ---- roofline of the dominant kernel family (largest share of the per-layer time) ----
     fam = max(("exact", "top1"), key=lambda n: sum_us[n])
-    if fam == "exact":
+    if not table:
+        roof = {"bound": None, "achieved": None, "peak": None, "unit": None, "kernel": None, "launches": 0}
+    elif fam == "exact":
         hb = [r for r in table if r["exact_bound"] == "hbm"]; tb = [r for r in table if r["exact_bound"] == "tensor"]
         if sum(r["exact_us"] for r in hb) >= sum(r["exact_us"] for r in tb):
             ach = sum(r["exact_bytes"] for r in hb) / sum(r["exact_us"] for r in hb) / 1e3
@@ -351,7 +353,7 @@ def main():
         ach = sum(r["top1_bytes"] for r in table) / sum_us["top1"] / 1e3
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "kernel": "top-1 select+gather", "launches": len(table)}
-    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["frac"] = roof["achieved"] / roof["peak"] if table else None
     roof["peak_source"] = peaks["source"]
     roof["traffic"] = None
 
@@ -406,7 +408,7 @@ def main():
         "roofline": roof, "cpu_baseline": cpu,
         "breakdown_us": {"streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
                          "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
-                         "top1_speedup_over_exact": sum_us["exact"] / sum_us["top1"]},
+                         "top1_speedup_over_exact": (sum_us["exact"] / sum_us["top1"]) if table else None},
         "paper_context": "paper reports >7% training wall-clock speedup (ResNet-20/VGG-19, Titan Xp, TF 1.13, cuDNN 7.4.2)",
     }
     if args.detail:

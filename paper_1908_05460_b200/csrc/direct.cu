@@ -6,8 +6,9 @@
 //
 // Register-tiled kernel.  A CTA owns a (TKT*OTK) x (TCT*OTC) block of (k, c) with all R*S filter
 // taps, and a contiguous range of work items; an item is one image's band of BP x BQ output pixels.
-// Per item the dY band is staged in shared memory pixel-major ([k-group][pixel][TKT]) and the X
-// window channel-minor ([row][col][c]), both as fp32.  The OTK*OTC "output threads" of a pixel
+// Per item the dY band ([k][pixel]) and the X window ([row][col][c]) are staged in shared memory
+// as fp32, two stages deep: fp32 inputs are copied with 16-byte cp.async while the previous item is
+// being consumed; other inputs are converted on the way in.  The OTK*OTC "output threads" of a pixel
 // group each keep TKT*TCT*R*S accumulators in registers; the 128/(OTK*OTC) pixel groups take the
 // band's pixels round-robin, so one vector load of dY and R*S vector loads of X feed
 // TKT*TCT*R*S FMAs.  At the end the pixel groups are summed (warp shuffles, then shared memory, in a
@@ -24,6 +25,17 @@ template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloa
     return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
 }
 
+// four consecutive elements as floats (16-byte load for fp32, 8-byte load for bf16)
+__device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void ld4(const __nv_bfloat16* p, float (&v)[4]) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
 constexpr int kThreads = 128;
 
 template <int N> struct Vec;
@@ -31,7 +43,83 @@ template <> struct Vec<1> { float v[1]; __device__ void load(const float* p) { v
 template <> struct Vec<2> { float v[2]; __device__ void load(const float* p) { float2 t = *reinterpret_cast<const float2*>(p); v[0] = t.x; v[1] = t.y; } };
 template <> struct Vec<4> { float v[4]; __device__ void load(const float* p) { float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; } };
 
-template <typename T, int R, int S, int TKT, int TCT, int OTK, int OTC>
+// 16-byte asynchronous global -> shared copy (fp32 fast path) and its group bookkeeping
+__device__ __forceinline__ void cp_async16(float* smem_dst, const float* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Stage one work item: dY band as [k][pixel] (row stride dys) and X window as [row][col][TC], fp32.
+// ASYNC (fp32 inputs, vector paths): 16-byte cp.async copies, zeros stored directly where the
+// tile leaves the tensor.  Otherwise: synchronous loads with conversion.
+template <typename T, bool ASYNC, int TK, int TC>
+__device__ __forceinline__ void stage_item(const T* __restrict__ x, const T* __restrict__ dy, float* s_dy, float* s_x,
+                                           const Geom& g, const DirectPlan& pl, int it, int k0, int c0, int dys,
+                                           int win_h, int win_w)
+{
+    const int npx = pl.bp * pl.bq;
+    const int n = it / (pl.bands_p * pl.bands_q);
+    const int band = it % (pl.bands_p * pl.bands_q);
+    const int p0 = (band / pl.bands_q) * pl.bp, q0 = (band % pl.bands_q) * pl.bq;
+    const int h0 = p0 * g.stride_h - g.pad_h, w0 = q0 * g.stride_w - g.pad_w;
+    if (pl.vec_dy) {
+        const int quads = npx >> 2;
+        for (int i = threadIdx.x; i < TK * quads; i += kThreads) {
+            const int kk = i / quads, j = (i - kk * quads) << 2, k = k0 + kk;
+            float* dst = s_dy + kk * dys + j;
+            const T* src = dy + ((long long)n * g.k + k) * g.p * g.q + (long long)p0 * g.q + j;
+            if constexpr (ASYNC) {
+                if (k < g.k) cp_async16(dst, reinterpret_cast<const float*>(src));
+                else *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                float v[4] = {0.f, 0.f, 0.f, 0.f};
+                if (k < g.k) ld4(src, v);
+                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < TK * npx; i += kThreads) {
+            const int kk = i / npx, j = i % npx;
+            const int p = p0 + j / pl.bq, q = q0 + j % pl.bq, k = k0 + kk;
+            float v = 0.f;
+            if (k < g.k && p < g.p && q < g.q) v = ldf(dy + (((long long)n * g.k + k) * g.p + p) * g.q + q);
+            s_dy[kk * dys + j] = v;
+        }
+    }
+    if (pl.vec_x) {
+        constexpr int CQ = TC / 4;                                // channel quads per pixel of the tile
+        for (int hh = 0; hh < win_h; ++hh) {
+            const int h = h0 + hh;
+            const bool row_ok = h >= 0 && h < g.h;
+            const T* xrow = x + n * g.xs_n + (long long)h * g.xs_h;
+            float* drow = s_x + hh * win_w * TC;
+            for (int i = threadIdx.x; i < win_w * CQ; i += kThreads) {
+                const int wq = i / CQ, cq = i - wq * CQ, ww = w0 + wq, c = c0 + 4 * cq;
+                const bool ok = row_ok && ww >= 0 && ww < g.w && c < g.c;
+                if constexpr (ASYNC) {
+                    if (ok) cp_async16(drow + i * 4, reinterpret_cast<const float*>(xrow + (long long)ww * g.xs_w + c));
+                    else *reinterpret_cast<float4*>(drow + i * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+                } else {
+                    float v[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (ok) ld4(xrow + (long long)ww * g.xs_w + c, v);
+                    *reinterpret_cast<float4*>(drow + i * 4) = make_float4(v[0], v[1], v[2], v[3]);
+                }
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < win_h * win_w * TC; i += kThreads) {
+            const int cc = i % TC, pix = i / TC;
+            const int hh = h0 + pix / win_w, ww = w0 + pix % win_w, c = c0 + cc;
+            float v = 0.f;
+            if (c < g.c && hh >= 0 && hh < g.h && ww >= 0 && ww < g.w)
+                v = ldf(x + n * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w);
+            s_x[i] = v;
+        }
+    }
+}
+
+template <typename T, bool ASYNC, int R, int S, int TKT, int TCT, int OTK, int OTC>
 __global__ void __launch_bounds__(kThreads)
 direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw,
                     float* __restrict__ partial, Geom g, DirectPlan pl)
@@ -40,9 +128,10 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
     static_assert(kThreads % OT == 0 && OT <= 64, "output threads must divide the CTA");
     extern __shared__ __align__(16) float smem[];
     const int npx = pl.bp * pl.bq;
+    const int dys = npx + 4;                     // row stride of the dY band: keeps rows 16-byte aligned, spreads banks
     const int win_h = (pl.bp - 1) * g.stride_h + R, win_w = (pl.bq - 1) * g.stride_w + S;
-    float* s_dy = smem;                          // [OTK][npx][TKT]
-    float* s_x = smem + TK * npx;                // [win_h][win_w][TC]
+    const int stage_floats = TK * dys + win_h * win_w * TC;   // a multiple of four
+    // two stages: the next item is fetched while the current one is consumed
 
     const int tile = blockIdx.x, split = blockIdx.y;
     const int k0 = (tile / pl.tiles_c) * TK, c0 = (tile % pl.tiles_c) * TC;
@@ -54,35 +143,30 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
     for (int i = 0; i < ACC; ++i) acc[i] = 0.f;
 
     const int per = (pl.items + pl.splits - 1) / pl.splits;
-    const int it_end = min(pl.items, (split + 1) * per);
-    for (int it = split * per; it < it_end; ++it) {
-        const int n = it / (pl.bands_p * pl.bands_q);
-        const int band = it % (pl.bands_p * pl.bands_q);
-        const int p0 = (band / pl.bands_q) * pl.bp, q0 = (band % pl.bands_q) * pl.bq;
-        __syncthreads();
-        // dY band: coalesced along pixels, stored as [k-group][pixel][TKT]
-        for (int i = threadIdx.x; i < TK * npx; i += kThreads) {
-            const int kk = i / npx, j = i % npx;
-            const int p = p0 + j / pl.bq, q = q0 + j % pl.bq, k = k0 + kk;
-            float v = 0.f;
-            if (k < g.k && p < g.p && q < g.q) v = ldf(dy + (((long long)n * g.k + k) * g.p + p) * g.q + q);
-            s_dy[((kk / TKT) * npx + j) * TKT + kk % TKT] = v;
-        }
-        const int h0 = p0 * g.stride_h - g.pad_h, w0 = q0 * g.stride_w - g.pad_w;
-        for (int i = threadIdx.x; i < win_h * win_w * TC; i += kThreads) {
-            const int cc = i % TC, pix = i / TC;
-            const int hh = h0 + pix / win_w, ww = w0 + pix % win_w, c = c0 + cc;
-            float v = 0.f;
-            if (c < g.c && hh >= 0 && hh < g.h && ww >= 0 && ww < g.w)
-                v = ldf(x + n * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w);
-            s_x[i] = v;
+    const int it_begin = split * per, it_end = min(pl.items, (split + 1) * per);
+    if (it_begin < it_end) {
+        stage_item<T, ASYNC, TK, TC>(x, dy, smem, smem + TK * dys, g, pl, it_begin, k0, c0, dys, win_h, win_w);
+        if (ASYNC) cp_async_commit();
+    }
+    int stage = 0;
+    for (int it = it_begin; it < it_end; ++it, stage ^= 1) {
+        float* cur = smem + stage * stage_floats;
+        if (it + 1 < it_end) {
+            float* nxt = smem + (stage ^ 1) * stage_floats;
+            stage_item<T, ASYNC, TK, TC>(x, dy, nxt, nxt + TK * dys, g, pl, it + 1, k0, c0, dys, win_h, win_w);
+            if (ASYNC) { cp_async_commit(); cp_async_wait<1>(); }
+        } else if (ASYNC) {
+            cp_async_wait<0>();
         }
         __syncthreads();
+        const float* s_dy = cur + otk * TKT * dys;
+        const float* s_x = cur + TK * dys + otc * TCT;
+        int pp = pg / pl.bq, qq = pg % pl.bq;
         for (int j = pg; j < npx; j += PG) {
-            const int pp = j / pl.bq, qq = j % pl.bq;
-            Vec<TKT> d;
-            d.load(s_dy + (otk * npx + j) * TKT);
-            const float* xb = s_x + ((pp * g.stride_h) * win_w + qq * g.stride_w) * TC + otc * TCT;
+            float d[TKT];
+#pragma unroll
+            for (int a = 0; a < TKT; ++a) d[a] = s_dy[a * dys + j];
+            const float* xb = s_x + ((pp * g.stride_h) * win_w + qq * g.stride_w) * TC;
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -93,9 +177,12 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
                     for (int a = 0; a < TKT; ++a)
 #pragma unroll
                         for (int b = 0; b < TCT; ++b)
-                            acc[((a * TCT + b) * R + r) * S + s] = fmaf(d.v[a], xv.v[b], acc[((a * TCT + b) * R + r) * S + s]);
+                            acc[((a * TCT + b) * R + r) * S + s] = fmaf(d[a], xv.v[b], acc[((a * TCT + b) * R + r) * S + s]);
                 }
+            qq += PG;
+            while (qq >= pl.bq) { qq -= pl.bq; ++pp; }
         }
+        __syncthreads();    // everyone is done with this stage before it is refilled
     }
 
     // ---- sum the pixel groups: lanes first (groups that share a warp), then warps through shared memory ----
@@ -163,6 +250,9 @@ direct_element_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* 
     dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * acc;
 }
 
+template <typename T> constexpr bool kAsyncOk = false;      // cp.async staging copies raw fp32
+template <> constexpr bool kAsyncOk<float> = true;
+
 // thread-tile shape of each variant
 struct Variant { int tkt, tct, otk, otc; };
 Variant variant_for(const Geom& g)
@@ -175,7 +265,7 @@ Variant variant_for(const Geom& g)
 size_t smem_for(const Geom& g, const Variant& v, int bp, int bq)
 {
     const int tk = v.tkt * v.otk, tc = v.tct * v.otc, ot = v.otk * v.otc;
-    const size_t stage = sizeof(float) * ((size_t)tk * bp * bq + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * tc);
+    const size_t stage = 2 * sizeof(float) * ((size_t)tk * (bp * bq + 4) + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * tc);
     const int sets = ot >= 32 ? kThreads / ot : kThreads / 32;
     const size_t red = sizeof(float) * (size_t)sets * ot * 16;
     return stage > red ? stage : red;
@@ -194,10 +284,17 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, const G
     const Variant v = variant_for(g);
     const size_t smem = smem_for(g, v, pl.bp, pl.bq);
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
+    const bool use_async = kAsyncOk<T> && pl.vec_dy && pl.vec_x;
     bool done = false;
 #define GACONV_DIRECT_CASE(RR, A, B, C, D)                                                                     \
     if (!done && g.r == RR && v.tkt == A && v.tct == B && v.otk == C && v.otc == D) {                          \
-        direct_tiled_kernel<T, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
+        if (use_async) {                                                                                       \
+            if (smem > 48 * 1024) cudaFuncSetAttribute(direct_tiled_kernel<T, kAsyncOk<T>, RR, RR, A, B, C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            direct_tiled_kernel<T, kAsyncOk<T>, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
+        } else {                                                                                               \
+            if (smem > 48 * 1024) cudaFuncSetAttribute(direct_tiled_kernel<T, false, RR, RR, A, B, C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            direct_tiled_kernel<T, false, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
+        }                                                                                                      \
         done = true;                                                                                           \
     }
     GACONV_DIRECT_CASE(1, 4, 4, 4, 4)
@@ -227,14 +324,19 @@ DirectPlan plan_direct(const Geom& g)
     pl.tiles_c = (g.c + tc - 1) / tc;
     pl.bq = g.q < 32 ? g.q : 32;
     pl.bp = 1;
-    while (pl.bp * 2 <= g.p && pl.bp * 2 * pl.bq <= 256 && smem_for(g, v, pl.bp * 2, pl.bq) <= 44 * 1024) pl.bp *= 2;
-    while (pl.bq > 1 && smem_for(g, v, pl.bp, pl.bq) > 44 * 1024) pl.bq /= 2;
+    while (pl.bp * 2 <= g.p && pl.bp * 2 * pl.bq <= 128 && smem_for(g, v, pl.bp * 2, pl.bq) <= 64 * 1024) pl.bp *= 2;
+    while (pl.bq > 1 && smem_for(g, v, pl.bp, pl.bq) > 64 * 1024) pl.bq /= 2;
     pl.bands_p = (g.p + pl.bp - 1) / pl.bp;
     pl.bands_q = (g.q + pl.bq - 1) / pl.bq;
+    // vector fast paths: bands of whole rows whose pixel runs start on a 4-element boundary; NHWC with
+    // channels a multiple of four (every 4-channel group is then aligned and entirely in or out of range)
+    pl.vec_dy = pl.bq == g.q && g.p % pl.bp == 0 && (pl.bp * g.q) % 4 == 0;
+    pl.vec_x = g.xs_c == 1 && g.c % 4 == 0 && tc % 4 == 0;
     pl.items = g.n * pl.bands_p * pl.bands_q;
     const int tiles = pl.tiles_k * pl.tiles_c;
-    // about three CTAs per SM; each split's partial block is written once and read once
-    int splits = (148 * 3 + tiles - 1) / tiles;
+    // one wave of two CTAs per SM (the register budget); each split's partial block is written once and read once
+    int splits = (148 * 2) / tiles;
+    if (splits < 1) splits = 1;
     if (splits > pl.items) splits = pl.items;
     const size_t out_bytes = (size_t)g.k * g.c * g.r * g.s * sizeof(float);
     while (splits > 1 && (size_t)splits * out_bytes > ((size_t)96 << 20)) --splits;

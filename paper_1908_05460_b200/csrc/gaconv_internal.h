@@ -61,6 +61,7 @@ struct DirectPlan {
     int splits;             // CTAs per output tile along the reduction
     size_t partial_bytes;
     bool tiled;             // false: filter size without a tiled instantiation -> per-element kernel
+    bool vec_dy, vec_x;     // 4-element vector loads usable for the dY band / the X window
 };
 DirectPlan plan_direct(const Geom& g);
 cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
