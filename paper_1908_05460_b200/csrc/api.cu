@@ -187,8 +187,10 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     if (x == nullptr || dy == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy)) return GACONV_ERR_MISALIGNED;
     const Top1Layout L = top1_layout(g);
-    st = check_ws(desc, L.total);
+    st = check_ws(desc, L.total);       // required by every route, so that behaviour does not depend on the kernel picked
     if (st != GACONV_OK) return st;
+    if (top1_fused_supported(g) && desc->algo != GACONV_ALGO_DIRECT)
+        return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     char* ws = static_cast<char*>(desc->workspace);
     int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx_off);
     float* sum = reinterpret_cast<float*>(ws + L.sum_off);

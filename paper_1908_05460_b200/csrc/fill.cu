@@ -31,9 +31,17 @@ __device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint
 
 __device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float& z0, float& z1)
 {
-    // ln in double: u1 close to 1 would lose all its information in fp32
-    const double u1 = ((double)wa + 1.0) * (1.0 / 4294967296.0);
-    const float rho = sqrtf((float)(-2.0 * log(u1)));
+    // ln u1 with u1 = (wa+1) 2^-32, in fp32 without losing u1 near 1: below one half take the
+    // logarithm of the (rounded) value itself -- a relative error of 2^-24 in u1 is an absolute error
+    // of 2^-24 in ln u1; above, 1-u1 = t 2^-32 with t an integer, and log1p keeps its relative accuracy.
+    float ln_u1;
+    if (wa < 0x7fffffffu) {
+        ln_u1 = logf((float)(wa + 1u) * (1.0f / 4294967296.0f));
+    } else {
+        const uint32_t t = 0xffffffffu - wa;                 // 2^32 - (wa+1)
+        ln_u1 = log1pf(-(float)t * (1.0f / 4294967296.0f));
+    }
+    const float rho = sqrtf(-2.0f * ln_u1);
     float sn, cs;
     sincospif(2.0f * ((float)wb * (1.0f / 4294967296.0f)), &sn, &cs);
     z0 = rho * cs; z1 = rho * sn;

@@ -48,6 +48,10 @@ GatherPlan plan_gather(const Geom& g);
 cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, float* dw, float* partial,
                           uint32_t* counters, const Geom& g, const GatherPlan& plan, cudaStream_t stream);
 
+// ---- Algorithm 1 in one launch (selection + patch accumulate + cluster reduction) ----
+bool top1_fused_supported(const Geom& g);
+cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream);
+
 // ---- zero / random gradient ----
 cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream);
 cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cudaStream_t stream);

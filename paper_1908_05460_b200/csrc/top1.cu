@@ -1,10 +1,14 @@
-// Max-gradient approximation (paper Section 2.3, Algorithm 1) as two kernels:
+// Max-gradient approximation (paper Section 2.3, Algorithm 1).  top1_fused_kernel does the whole method
+// in one launch (thread-block clusters, distributed shared memory); the two-kernel form below is kept
+// for shapes whose per-channel block does not fit shared memory and for the inspection entry point:
 //   select_kernel  -- per (n,k) map of dY: position of the largest magnitude (lowest index among
 //                     equals) and the signed sum of the map      [Algorithm 1, arg-max and sum lines]
 //   gather_kernel  -- dW[k,r,s,c] = alpha * sum_n sum[n,k] * Xz[n, c, patch at the selected position]
 //                                                                  [Algorithm 1, accumulation line]
 // Selection compares the bit pattern of |v| in the input dtype as an unsigned integer, which orders
 // finite values exactly as their magnitudes do, so indices are reproducible bit for bit.
+#include <cooperative_groups.h>
+
 #include "gaconv_internal.h"
 
 namespace gaconv {
@@ -65,21 +69,15 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     return v;
 }
 
-// One group of G lanes (G a power of two, G <= 32) scans one map.  VEC: 16-byte loads (maps are a
-// whole number of 16-byte vectors and therefore 16-byte aligned) or element loads.
+// A group of G lanes (G a power of two, G <= 32) scans one map: each lane takes every G-th 16-byte
+// vector (VEC: maps are a whole number of vectors, hence 16-byte aligned) or every G-th element, keeps
+// its first largest magnitude and its running sum; the lanes are then combined -- larger magnitude
+// wins, then the lower index; sums add in a fixed tree.  All 32 lanes of the warp must call this.
 template <typename T, bool VEC>
-__global__ void __launch_bounds__(256)
-select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __restrict__ sum,
-              T* __restrict__ dy_sparse, long long num_maps, int pq, int G)
+__device__ __forceinline__ void scan_map(const T* __restrict__ map, bool live, int pq, int G, int sub,
+                                         int& best_j, float& sum)
 {
-    const int lane = threadIdx.x & 31;
-    const int sub = lane & (G - 1);
-    const int maps_per_warp = 32 / G;
-    const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const long long m = warp * maps_per_warp + lane / G;
-    const bool live = m < num_maps;
     Scan sc{-1, 0, 0.0f};
-    const T* map = dy + (live ? m : 0) * (long long)pq;
     if (live) {
         if (VEC) {
             constexpr int E = Elem<T>::kPerVec;
@@ -100,7 +98,6 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
             for (int j = sub; j < pq; j += G) Elem<T>::visit1(map, j, sc);
         }
     }
-    // combine the G lanes: larger magnitude wins, then the lower index; sums add in a fixed tree
     unsigned long long key = ((unsigned long long)(unsigned)(sc.best_mag + 1) << 32) | (0xffffffffu - (unsigned)sc.best_j);
     float s = sc.sum;
     for (int off = G >> 1; off > 0; off >>= 1) {
@@ -109,8 +106,24 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
         key = other > key ? other : key;
         s += so;
     }
+    best_j = (int)(0xffffffffu - (unsigned)(key & 0xffffffffu));
+    sum = s;
+}
+
+// Selection alone (inspection entry point): idx, sum and optionally the dense sparse tensor.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(256)
+select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __restrict__ sum,
+              T* __restrict__ dy_sparse, long long num_maps, int pq, int G)
+{
+    const int lane = threadIdx.x & 31;
+    const int sub = lane & (G - 1);
+    const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long m = warp * (32 / G) + lane / G;
+    const bool live = m < num_maps;
+    int best_j; float s;
+    scan_map<T, VEC>(dy + (live ? m : 0) * (long long)pq, live, pq, G, sub, best_j, s);
     if (!live) return;
-    const int best_j = (int)(0xffffffffu - (unsigned)(key & 0xffffffffu));
     if (sub == 0) { idx[m] = best_j; sum[m] = s; }
     if (dy_sparse != nullptr) {
         T* out = dy_sparse + m * (long long)pq;
@@ -118,10 +131,131 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
     }
 }
 
+// four consecutive elements as floats (16-byte load for fp32, 8-byte load for bf16)
+__device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void ld4(const __nv_bfloat16* p, float (&v)[4]) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
 template <typename T> __device__ __forceinline__ float ld_as_float(const T* p);
 template <> __device__ __forceinline__ float ld_as_float<float>(const float* p) { return __ldg(p); }
 template <> __device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __nv_bfloat16* p) {
     return bf16_bits_to_float(__ldg(reinterpret_cast<const unsigned short*>(p)));
+}
+
+// Algorithm 1 in one launch.  grid (CL, K), thread-block clusters of CL CTAs along x: the CL CTAs of
+// a cluster share one output channel k and split the batch into CL contiguous ranges of images.
+//   phase 1  each CTA scans the dY maps of its images (selection),
+//   phase 2  accumulates their patches, images in order, into a shared-memory block of R*S*C sums,
+//   phase 3  after a cluster barrier, CTA j adds slice j of the block over the CL CTAs through
+//            distributed shared memory, in rank order, and writes alpha * total to dW.
+// No global scratch, no atomics; the order of every sum is fixed.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(256, 4)
+top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int rsc = g.r * g.s * g.c;
+    float* s_part = reinterpret_cast<float*>(smem_raw);                 // [rsc]
+    int* s_h0 = reinterpret_cast<int*>(s_part + rsc);                   // [ipc] top-left input row of each patch
+    int* s_w0 = s_h0 + ipc;
+    float* s_sum = reinterpret_cast<float*>(s_w0 + ipc);
+
+    const int k = blockIdx.y, chunk = blockIdx.x, CL = gridDim.x;
+    const int n0 = chunk * ipc;
+    const int cnt = max(0, min(ipc, g.n - n0));
+    const int pq = g.p * g.q;
+
+    // ---- phase 1: selection ----
+    {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const int sub = lane & (G - 1), per_warp = 32 / G, per_pass = (blockDim.x >> 5) * per_warp;
+        for (int base = 0; base < cnt; base += per_pass) {
+            const int i = base + warp * per_warp + lane / G;
+            const bool live = i < cnt;
+            int best_j; float s;
+            scan_map<T, VEC>(dy + ((long long)(n0 + (live ? i : 0)) * g.k + k) * pq, live, pq, G, sub, best_j, s);
+            if (live && sub == 0) {
+                s_h0[i] = (best_j / g.q) * g.stride_h - g.pad_h;
+                s_w0[i] = (best_j % g.q) * g.stride_w - g.pad_w;
+                s_sum[i] = s;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- phase 2: patch accumulate ----
+    // A work item is (element group, image lane j): NJ lanes split the images round-robin
+    // (i = j, j+NJ, ...), each adding its images in ascending order with up to eight loads in flight;
+    // the NJ subtotals are then added in lane order.  VX elements per group: four channels per load
+    // on the vector path (NHWC, C a multiple of four), else one.
+    {
+        const int VX = vec_x ? 4 : 1;
+        const int groups = rsc / VX;
+        int NJ = 1;
+        while (NJ * 2 * groups <= (int)blockDim.x && NJ * 2 <= 16) NJ *= 2;
+        float* s_sub = s_part;                                  // NJ == 1: results go straight to s_part
+        if (NJ > 1) s_sub = reinterpret_cast<float*>(s_sum + ipc);   // [NJ][rsc] scratch after the per-image arrays
+        for (int item = threadIdx.x; item < groups * NJ; item += blockDim.x) {
+            const int j = item / groups, e = (item - j * groups) * VX;
+            const int c = e % g.c, rs = e / g.c, s = rs % g.s, r = rs / g.s;
+            const T* xc = x + n0 * g.xs_n + c * g.xs_c;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int i0 = j; i0 < cnt; i0 += 8 * NJ) {
+                float v[8][4];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + u * NJ;
+                    const int hh = (i < cnt ? s_h0[i] : -1) + r, ww = (i < cnt ? s_w0[i] : -1) + s;
+                    const bool ok = i < cnt && hh >= 0 && hh < g.h && ww >= 0 && ww < g.w;
+                    const long long off = ok ? i * g.xs_n + hh * g.xs_h + ww * g.xs_w : 0;   // element 0 is always readable
+                    if (vec_x) ld4(xc + off, v[u]);
+                    else { v[u][0] = ld_as_float(xc + off); v[u][1] = v[u][2] = v[u][3] = 0.f; }
+                    if (!ok) v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + u * NJ;
+                    if (i < cnt) {
+                        const float sm_ = s_sum[i];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) acc[t] = fmaf(sm_, v[u][t], acc[t]);
+                    }
+                }
+            }
+            for (int t = 0; t < VX; ++t) s_sub[j * rsc + e + t] = acc[t];
+        }
+        if (NJ > 1) {
+            __syncthreads();
+            for (int e = threadIdx.x; e < rsc; e += blockDim.x) {
+                float tot = s_sub[e];
+                for (int j = 1; j < NJ; ++j) tot += s_sub[j * rsc + e];
+                s_part[e] = tot;
+            }
+        }
+    }
+    cluster.sync();
+
+    // ---- phase 3: rank j finishes slice j ----
+    const int slice = (rsc + CL - 1) / CL;
+    const int e_end = min(rsc, (chunk + 1) * slice);
+    for (int e = chunk * slice + threadIdx.x; e < e_end; e += blockDim.x) {
+        float pv[8];
+#pragma unroll
+        for (int rk = 0; rk < 8; ++rk) pv[rk] = rk < CL ? *cluster.map_shared_rank(s_part + e, rk) : 0.0f;
+        float tot = 0.0f;
+#pragma unroll
+        for (int rk = 0; rk < 8; ++rk) tot += pv[rk];          // rank order; absent ranks add +0
+        const int c = e % g.c, rs = e / g.c, s = rs % g.s, r = rs / g.s;
+        dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * tot;
+    }
+    cluster.sync();     // peers may still be reading this CTA's block
 }
 
 // grid (chunks, K).  Each CTA owns the images [chunk*ipc, (chunk+1)*ipc) of one output channel and
@@ -186,6 +320,18 @@ gather_kernel(const T* __restrict__ x, const int32_t* __restrict__ idx, const fl
 
 int pow2_floor(int v) { int p = 1; while (p * 2 <= v) p *= 2; return p; }
 
+struct MapScanShape { bool vec; int G; };
+MapScanShape map_scan_shape(const Geom& g)
+{
+    const int pq = g.p * g.q, eb = g.bf16 ? 2 : 4;
+    MapScanShape m;
+    m.vec = ((size_t)pq * eb) % 16 == 0;
+    const int units = m.vec ? pq * eb / 16 : pq;
+    m.G = pow2_floor(units);
+    if (m.G > 32) m.G = 32;
+    return m;
+}
+
 }  // namespace
 
 cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_sparse, const Geom& g,
@@ -193,20 +339,17 @@ cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_spa
 {
     const long long maps = (long long)g.n * g.k;
     const int pq = g.p * g.q;
-    const int eb = g.bf16 ? 2 : 4;
-    const bool vec = ((size_t)pq * eb) % 16 == 0;
-    const int units = vec ? pq * eb / 16 : pq;
-    int G = pow2_floor(units); if (G > 32) G = 32;
-    const int maps_per_cta = (256 / 32) * (32 / G);
+    const MapScanShape m = map_scan_shape(g);
+    const int maps_per_cta = (256 / 32) * (32 / m.G);
     const unsigned grid = (unsigned)((maps + maps_per_cta - 1) / maps_per_cta);
     if (g.bf16) {
         auto d = static_cast<const __nv_bfloat16*>(dy); auto o = static_cast<__nv_bfloat16*>(dy_sparse);
-        if (vec) select_kernel<__nv_bfloat16, true><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
-        else     select_kernel<__nv_bfloat16, false><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
+        if (m.vec) select_kernel<__nv_bfloat16, true><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, m.G);
+        else       select_kernel<__nv_bfloat16, false><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, m.G);
     } else {
         auto d = static_cast<const float*>(dy); auto o = static_cast<float*>(dy_sparse);
-        if (vec) select_kernel<float, true><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
-        else     select_kernel<float, false><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, G);
+        if (m.vec) select_kernel<float, true><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, m.G);
+        else       select_kernel<float, false><<<grid, 256, 0, stream>>>(d, idx, sum, o, maps, pq, m.G);
     }
     note_launch();
     return cudaGetLastError();
@@ -240,6 +383,60 @@ cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, f
                                                           counters, g, plan.chunks, plan.imgs_per_chunk);
     note_launch();
     return cudaGetLastError();
+}
+
+bool top1_fused_supported(const Geom& g)
+{
+    // the per-channel block of R*S*C sums lives in shared memory
+    return (size_t)g.r * g.s * g.c * sizeof(float) <= 160 * 1024 && g.k <= 65535;
+}
+
+template <typename T, bool VEC>
+static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom& g, int cl, int ipc, int G, cudaStream_t stream)
+{
+    // block of sums + per-image arrays + up to 16 lane subtotals when the block is small
+    const int rsc = g.r * g.s * g.c;
+    const bool vec_x = g.xs_c == 1 && g.c % 4 == 0;
+    int nj = 1;
+    while (nj * 2 * (rsc / (vec_x ? 4 : 1)) <= 256 && nj * 2 <= 16) nj *= 2;
+    const size_t smem = (size_t)rsc * sizeof(float) * (nj > 1 ? 1 + nj : 1) + (size_t)ipc * 12 + 16;
+    static size_t configured = 0;
+    if (smem > 48 * 1024 && smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(top1_fused_kernel<T, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cl, g.k);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, top1_fused_kernel<T, VEC>, x, dy, dw, g, ipc, G, vec_x);
+    note_launch();
+    return e;
+}
+
+cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream)
+{
+    int cl = 1;
+    while (cl * 2 <= 8 && cl * 2 <= g.n) cl *= 2;
+    // fewer, fatter CTAs when there are already plenty of channels: the whole grid should be resident
+    // at once (clusters are placed GPC by GPC), i.e. about two CTAs per SM
+    while (cl > 1 && (long long)cl * g.k > 148 * 2) cl /= 2;
+    const int ipc = (g.n + cl - 1) / cl;
+    const MapScanShape m = map_scan_shape(g);
+    if (g.bf16) {
+        auto xx = static_cast<const __nv_bfloat16*>(x); auto dd = static_cast<const __nv_bfloat16*>(dy);
+        return m.vec ? launch_fused_t<__nv_bfloat16, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
+                     : launch_fused_t<__nv_bfloat16, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
+    }
+    auto xx = static_cast<const float*>(x); auto dd = static_cast<const float*>(dy);
+    return m.vec ? launch_fused_t<float, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
+                 : launch_fused_t<float, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
 }
 
 }  // namespace gaconv

@@ -71,7 +71,9 @@ def test_top1_matches_oracle(li, dtype):
     np.put_along_axis(want, idx_ref[..., None].astype(np.int64),
                       torch.from_numpy(s).to(dtype).to(torch.float64).numpy()[..., None], axis=2)
     np.testing.assert_array_equal(sp, want)
-    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
+    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)                  # one-launch cluster kernel
+    g2 = GpuLayer(layer, dtype, x, dy, alpha=1.0 / 128, algo=B.ALGO_DIRECT)
+    assert norm_err(g2.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)                 # select + gather kernels
 
 
 @pytest.mark.parametrize("x_layout,dw_layout", [(B.X_NCHW, B.DW_KCRS), (B.X_NHWC, B.DW_KCRS), (B.X_NCHW, B.DW_KRSC)])
