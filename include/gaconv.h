@@ -95,6 +95,29 @@ gaconv_status_t gaconv_workspace_init(void *workspace, size_t bytes, void *strea
 gaconv_status_t gaconv_dw_exact(const void *x, const void *dy, float *dw,
                                 const gaconv_conv_desc_t *desc, void *stream);
 
+/* gaconv_dw_exact for callers that cannot allocate device memory (no counterpart in the paper).
+ * Some callers cannot give the library a workspace because they may not call cudaMalloc where they
+ * run: a host framework's plugin that is handed only its inputs and outputs, a loop that was promised
+ * "no allocation after warm-up", a process whose device memory pool belongs to someone else.  This
+ * variant computes exactly what gaconv_dw_exact computes, with the same kernels, but keeps the scratch
+ * (split partial sums, control words) in a fixed array inside the library: gaconv_static_scratch_bytes()
+ * bytes (8 MiB) that every GPU loading the library holds until the process exits.  desc->workspace and
+ * desc->workspace_bytes are ignored.  The call allocates nothing (no cudaMalloc, cudaFree or
+ * allocating library routine).
+ *   - Limit: a problem whose gaconv_workspace_size(desc, GACONV_METHOD_EXACT) exceeds
+ *     gaconv_static_scratch_bytes() is rejected with GACONV_ERR_WORKSPACE_TOO_SMALL and nothing is
+ *     enqueued; use gaconv_dw_exact with a caller-owned workspace for those.
+ *   - The first call on each device resolves the array's device address and clears its control words
+ *     on `stream`; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents (each call
+ *     overwrites what it later reads).  Calls that can overlap on the GPU (different streams without
+ *     ordering between them) race on it: serialise them, or use gaconv_dw_exact with separate
+ *     workspaces.
+ * Other errors as gaconv_dw_exact. */
+gaconv_status_t gaconv_dw_exact_static(const void *x, const void *dy, float *dw,
+                                       const gaconv_conv_desc_t *desc, void *stream);
+size_t gaconv_static_scratch_bytes(void);
+
 /* Approximated filter gradient, Section 2:
  *   GACONV_METHOD_ZERO   (2.1)  dw = +0.
  *   GACONV_METHOD_RANDOM (2.2)  dw[i] = rand_std * z_i, z_i independent standard normals drawn from

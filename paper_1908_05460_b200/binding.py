@@ -32,6 +32,7 @@ EXPORTS = [
     "gaconv_status_string", "gaconv_launch_count", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
     "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_poll_async_status",
     "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_destroy",
+    "gaconv_dw_exact_static", "gaconv_static_scratch_bytes",
 ]
 
 
@@ -70,6 +71,9 @@ def load():
     lib.gaconv_workspace_size.argtypes = [dp, i32, ctypes.POINTER(sz)]
     lib.gaconv_workspace_init.argtypes = [vp, sz, vp]
     lib.gaconv_dw_exact.argtypes = [vp, vp, vp, dp, vp]
+    lib.gaconv_dw_exact_static.argtypes = [vp, vp, vp, dp, vp]
+    lib.gaconv_static_scratch_bytes.restype = sz
+    lib.gaconv_static_scratch_bytes.argtypes = []
     lib.gaconv_dw_approx.argtypes = [i32, vp, vp, vp, dp, u64, vp]
     lib.gaconv_approx_select.argtypes = [vp, vp, vp, vp, dp, vp]
     lib.gaconv_dw_from_host.argtypes = [i32, vp, vp, vp, vp, vp, vp, dp, u64, vp]
@@ -150,6 +154,18 @@ def attach_workspace(desc: ConvDesc, methods=(METHOD_EXACT, METHOD_TOP1), device
 
 def gaconv_dw_exact(x, dy, dw, desc: ConvDesc, stream=None):
     _check(load().gaconv_dw_exact(_ptr(x), _ptr(dy), _ptr(dw), ctypes.byref(desc), _stream(stream)), "gaconv_dw_exact")
+
+
+def gaconv_dw_exact_static(x, dy, dw, desc: ConvDesc, stream=None):
+    """Exact dW for callers that cannot allocate: scratch lives in a fixed array inside the library
+    (gaconv_static_scratch_bytes() per GPU); desc.workspace is ignored.  Raises GaconvError with
+    ERR_WORKSPACE_TOO_SMALL when the problem needs more scratch than that array holds."""
+    _check(load().gaconv_dw_exact_static(_ptr(x), _ptr(dy), _ptr(dw), ctypes.byref(desc), _stream(stream)),
+           "gaconv_dw_exact_static")
+
+
+def gaconv_static_scratch_bytes() -> int:
+    return int(load().gaconv_static_scratch_bytes())
 
 
 def gaconv_dw_approx(method: int, x, dy, dw, desc: ConvDesc, seed: int = 0, stream=None):
