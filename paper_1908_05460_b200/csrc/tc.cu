@@ -16,7 +16,9 @@
 // A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks; the
 // partial blocks of the splits are summed in split order by a second, element-parallel kernel.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue.
+// Warp roles: warp 0 = TMA producer; warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns
+// the TMEM allocation); warps 4..7 = epilogue.  The filter rows are dealt round-robin to the issuers:
+// a single thread sustains only one small MMA per ~60 cycles, and rows accumulate independently.
 // Every mbarrier wait is bounded; on expiry the kernel raises the workspace status word, drains
 // the copies it has in flight, frees its tensor memory and returns.
 #include <cuda.h>
@@ -106,6 +108,7 @@ struct TcParams {
     int stage_bytes, stages;
     int ksteps;         // ci*bp*Q/16
     int tmem_cols;      // power of two >= 32
+    int issuers;        // MMA-issuing warps: min(R, 3); issuer i takes filter rows i, i+issuers, ...
     uint32_t idesc;
     int timeline;       // 1: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
 };
@@ -115,7 +118,7 @@ constexpr int kMaxStages = 8;
 // R_T: filter rows (0 = take it from the geometry); KS_T: k-steps per A box (0 = from the plan).
 // The compile-time values let the issue loop unroll into straight-line MMA instructions.
 template <int R_T, int KS_T>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(256, 1)
 exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
                 float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters,
                 uint32_t* __restrict__ status, const TcParams P)
@@ -137,8 +140,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int nmma = g.s * P.ct;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
-        mbar_init(smem_u32(&bar_acc), 1);
+        for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), P.issuers); }
+        mbar_init(smem_u32(&bar_acc), P.issuers);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -191,7 +194,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         if (s_abort) {   // drain: wait (bounded) for the copies already issued
             for (int it = max(0, issued - P.stages); it < issued; ++it) mbar_wait(smem_u32(&bar_full[it % P.stages]), (it / P.stages) & 1);
         }
-    } else if (warp == 1 && lane == 0) {
+    } else if (warp >= 1 && warp <= 3 && warp - 1 < P.issuers && lane == 0) {
+        const int issuer = warp - 1;
         // ------------------------------------------------------------------ MMA issuer
         // descriptors are assembled from a constant high word and a low word that only advances
         const uint32_t a_row_bytes = P.a_sub_px * 2, b_row_bytes = P.ct * 2;
@@ -201,10 +205,19 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const int ks_per_sub = P.a_sub_px / 16;
         const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4, b_k_step = (16 * b_row_bytes) >> 4;
         const uint32_t b_r_step = (P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
-        const uint32_t d_step_even = P.m == 128 ? (uint32_t)nmma : (16u << 16);                 // r -> r+1, r even
-        const uint32_t d_step_odd = P.m == 128 ? (uint32_t)nmma : (uint32_t)nmma - (16u << 16);  // r -> r+1, r odd
         const int R = R_T ? R_T : g.r;
         const int KS = KS_T ? KS_T : ks_per_sub;
+        // this issuer's filter rows: TMEM address of the accumulator and descriptor offset of the row
+        constexpr int RI = R_T == 0 ? 3 : (R_T + 2) / 3;           // rows per issuer, at most (R <= 7 -> 3)
+        uint32_t d_row[RI], b_row[RI];
+        int nrows = 0;
+#pragma unroll
+        for (int i = 0; i < RI; ++i) {
+            const int r = issuer + i * P.issuers;
+            d_row[i] = P.m == 128 ? tmem_base + r * nmma : tmem_base + (((uint32_t)(r & 1) * 16u) << 16) + (r >> 1) * nmma;
+            b_row[i] = r * b_r_step;
+            if (r < R) nrows = i + 1;
+        }
         const uint64_t a_hi64 = (uint64_t)a_hi << 32, b_hi64 = (uint64_t)b_hi << 32;
         const uint32_t idesc = P.idesc;
         int st = 0, ph = 0;
@@ -212,28 +225,22 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         for (int it = 0; it < nchunks; ++it) {
             if (!mbar_wait(smem_u32(&bar_full[st]), ph)) { s_abort = 1; atomicOr(status, 1u); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (tl && it == 0) tl[1] = clock64();
+            if (tl && it == 0 && issuer == 0) tl[1] = clock64();
             const uint32_t sa = smem_base + st * P.stage_bytes;
             uint32_t a_lo = a_lo_c | (sa >> 4);
             uint32_t b_lo = b_lo_c | ((sa + P.a_region_bytes) >> 4);
             for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
                 if (fresh) {      // first k-step of this CTA: accumulate flag off
-                    uint32_t d = tmem_base, bl = b_lo;
 #pragma unroll
-                    for (int r = 0; r < R; ++r, bl += b_r_step) {
-                        umma_bf16(d, a_hi64 | a_lo, b_hi64 | bl, idesc, 0u);
-                        d += (r & 1) ? d_step_odd : d_step_even;
-                    }
+                    for (int i = 0; i < RI; ++i)
+                        if (i < nrows) umma_bf16(d_row[i], a_hi64 | a_lo, b_hi64 | (b_lo + b_row[i]), idesc, 0u);
                 }
 #pragma unroll
                 for (int k4 = 0; k4 < KS; ++k4) {
                     if (!(fresh && k4 == 0)) {
-                        uint32_t d = tmem_base, bl = b_lo + k4 * b_k_step;
 #pragma unroll
-                        for (int r = 0; r < R; ++r, bl += b_r_step) {
-                            umma_bf16_acc(d, a_hi64 | (a_lo + 2 * k4), b_hi64 | bl, idesc);
-                            d += (r & 1) ? d_step_odd : d_step_even;
-                        }
+                        for (int i = 0; i < RI; ++i)
+                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + 2 * k4), b_hi64 | (b_lo + k4 * b_k_step + b_row[i]), idesc);
                     }
                 }
                 fresh = false;
@@ -243,13 +250,13 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             if (++st == P.stages) { st = 0; ph ^= 1; }
         }
         umma_commit(smem_u32(&bar_acc));             // accumulators complete
-        if (tl) tl[2] = clock64();
-    } else if (warp >= 2) {
+        if (tl && issuer == 0) tl[2] = clock64();
+    } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue: TMEM -> global
         const bool ready = mbar_wait_sleepy(smem_u32(&bar_acc), 0);
         if (!ready) { s_abort = 1; atomicOr(status, 1u); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (tl && threadIdx.x == 64) tl[3] = clock64();
+        if (tl && threadIdx.x == 128) tl[3] = clock64();
         if (ready && !s_abort) {
             const int sp = warp & 3;
             float* out = P.splits == 1 ? dw : partial + (size_t)split * g.k * g.r * g.s * g.c;
@@ -296,7 +303,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         }
     }
 
-    if (tl && threadIdx.x == 64) tl[4] = clock64();
+    if (tl && threadIdx.x == 128) tl[4] = clock64();
     // ---------------------------------------------------------------------- teardown
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -345,7 +352,10 @@ bool plan_tc(const Geom& g, TcPlan* out)
 
     TcParams P{};
     P.g = g;
-    P.m = g.k <= 64 ? 64 : 128;
+    // M = 64 keeps two accumulators per TMEM column set, which is what lets a 64-channel tile (128-byte
+    // rows, the fast MN-major format) hold all three filter rows; M = 128 with 32-channel tiles measured
+    // about twice slower per FLOP, so it is used only where the tile is narrow anyway.
+    P.m = (g.k <= 64 || g.c >= 64) ? 64 : 128;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     // channels per tile: one swizzle span wide (16, 32 or 64 channels), limited by MMA N <= 256 and TMEM columns
     int ct = g.c >= 64 ? 64 : g.c >= 32 ? 32 : 16;
@@ -394,6 +404,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.stages = smem_budget / P.stage_bytes;
     if (P.stages > kMaxStages) P.stages = kMaxStages;
     if (P.stages < 2) return false;
+    P.issuers = g.r < 3 ? g.r : 3;
     P.tmem_cols = pow2_ceil(cols_for(ct));
     if (P.tmem_cols > 512) return false;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
@@ -468,7 +479,7 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
             if (err == cudaSuccess) configured = smem;                                                             \
         }                                                                                                          \
         if (err == cudaSuccess)                                                                                    \
-            exact_tc_kernel<RR, KK><<<grid, 192, smem, stream>>>(map_dy, map_x, dw, partial, counters, status, P);  \
+            exact_tc_kernel<RR, KK><<<grid, 256, smem, stream>>>(map_dy, map_x, dw, partial, counters, status, P);  \
     }
     GACONV_TC_CASE(3, 4)
     GACONV_TC_CASE(3, 1)
