@@ -165,7 +165,7 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
         return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
-                                  reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.dp,
+                                  reinterpret_cast<uint32_t*>(ws), g, L.dp,
                                   static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
 }

@@ -7,14 +7,15 @@
 // Register-tiled kernel.  A CTA owns a (TKT*OTK) x (TCT*OTC) block of (k, c) with all R*S filter
 // taps, and a contiguous range of work items; an item is one image's band of BP x BQ output pixels.
 // Per item the dY band ([k][pixel]) and the X window ([row][col][c]) are staged in shared memory
-// as fp32, two stages deep: fp32 inputs are copied with 16-byte cp.async while the previous item is
-// being consumed; other inputs are converted on the way in.  The OTK*OTC "output threads" of a pixel
+// as fp32, two stages deep: fp32 NHWC inputs arrive as TMA boxes (zero fill = padding) while the
+// previous item is being consumed; other inputs are loaded and converted by the threads.  The OTK*OTC "output threads" of a pixel
 // group each keep TKT*TCT*R*S accumulators in registers; the 128/(OTK*OTC) pixel groups take the
 // band's pixels round-robin, so one vector load of dY and R*S vector loads of X feed
 // TKT*TCT*R*S FMAs.  At the end the pixel groups are summed (warp shuffles, then shared memory, in a
 // fixed order) and the CTA writes its block: to dW if it is the only split, else to its slot of
 // the partial buffer, which reduce_splits() adds up in split order.
 #include "gaconv_internal.h"
+#include "tma.cuh"
 
 namespace gaconv {
 namespace {
@@ -43,17 +44,9 @@ template <> struct Vec<1> { float v[1]; __device__ void load(const float* p) { v
 template <> struct Vec<2> { float v[2]; __device__ void load(const float* p) { float2 t = *reinterpret_cast<const float2*>(p); v[0] = t.x; v[1] = t.y; } };
 template <> struct Vec<4> { float v[4]; __device__ void load(const float* p) { float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; } };
 
-// 16-byte asynchronous global -> shared copy (fp32 fast path) and its group bookkeeping
-__device__ __forceinline__ void cp_async16(float* smem_dst, const float* gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// Stage one work item: dY band as [k][pixel] (row stride dys) and X window as [row][col][TC], fp32.
-// ASYNC (fp32 inputs, vector paths): 16-byte cp.async copies, zeros stored directly where the
-// tile leaves the tensor.  Otherwise: synchronous loads with conversion.
-template <typename T, bool ASYNC, int TK, int TC>
+// Stage one work item with the CTA's threads: dY band as [k][pixel] (row stride dys) and X window as
+// [row][col][TC], converted to fp32; four elements per load where the layout allows.
+template <typename T, bool UNUSED, int TK, int TC>
 __device__ __forceinline__ void stage_item(const T* __restrict__ x, const T* __restrict__ dy, float* s_dy, float* s_x,
                                            const Geom& g, const DirectPlan& pl, int it, int k0, int c0, int dys,
                                            int win_h, int win_w)
@@ -69,14 +62,9 @@ __device__ __forceinline__ void stage_item(const T* __restrict__ x, const T* __r
             const int kk = i / quads, j = (i - kk * quads) << 2, k = k0 + kk;
             float* dst = s_dy + kk * dys + j;
             const T* src = dy + ((long long)n * g.k + k) * g.p * g.q + (long long)p0 * g.q + j;
-            if constexpr (ASYNC) {
-                if (k < g.k) cp_async16(dst, reinterpret_cast<const float*>(src));
-                else *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
-            } else {
-                float v[4] = {0.f, 0.f, 0.f, 0.f};
-                if (k < g.k) ld4(src, v);
-                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-            }
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            if (k < g.k) ld4(src, v);
+            *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
         }
     } else {
         for (int i = threadIdx.x; i < TK * npx; i += kThreads) {
@@ -97,14 +85,9 @@ __device__ __forceinline__ void stage_item(const T* __restrict__ x, const T* __r
             for (int i = threadIdx.x; i < win_w * CQ; i += kThreads) {
                 const int wq = i / CQ, cq = i - wq * CQ, ww = w0 + wq, c = c0 + 4 * cq;
                 const bool ok = row_ok && ww >= 0 && ww < g.w && c < g.c;
-                if constexpr (ASYNC) {
-                    if (ok) cp_async16(drow + i * 4, reinterpret_cast<const float*>(xrow + (long long)ww * g.xs_w + c));
-                    else *reinterpret_cast<float4*>(drow + i * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-                } else {
-                    float v[4] = {0.f, 0.f, 0.f, 0.f};
-                    if (ok) ld4(xrow + (long long)ww * g.xs_w + c, v);
-                    *reinterpret_cast<float4*>(drow + i * 4) = make_float4(v[0], v[1], v[2], v[3]);
-                }
+                float v[4] = {0.f, 0.f, 0.f, 0.f};
+                if (ok) ld4(xrow + (long long)ww * g.xs_w + c, v);
+                *reinterpret_cast<float4*>(drow + i * 4) = make_float4(v[0], v[1], v[2], v[3]);
             }
         }
     } else {
@@ -119,19 +102,25 @@ __device__ __forceinline__ void stage_item(const T* __restrict__ x, const T* __r
     }
 }
 
-template <typename T, bool ASYNC, int R, int S, int TKT, int TCT, int OTK, int OTC>
+// STAGING: 0 = loads by the threads with conversion (any dtype/layout); 1 = TMA tiles (fp32, NHWC,
+// C and P*Q multiples of four): one thread issues a 3-D box of dY and a 4-D box of X per item (zero
+// fill outside the tensor gives the padding) and an mbarrier per stage signals arrival.
+template <typename T, int STAGING, int R, int S, int TKT, int TCT, int OTK, int OTC>
 __global__ void __launch_bounds__(kThreads)
 direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw,
-                    float* __restrict__ partial, Geom g, DirectPlan pl)
+                    float* __restrict__ partial, uint32_t* __restrict__ status,
+                    const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
+                    Geom g, DirectPlan pl)
 {
     constexpr int TK = TKT * OTK, TC = TCT * OTC, OT = OTK * OTC, PG = kThreads / OT, ACC = TKT * TCT * R * S;
     static_assert(kThreads % OT == 0 && OT <= 64, "output threads must divide the CTA");
-    extern __shared__ __align__(16) float smem[];
+    extern __shared__ __align__(128) float smem[];
+    __shared__ __align__(8) uint64_t bar_full[2];
+    __shared__ volatile int s_fail;
     const int npx = pl.bp * pl.bq;
-    const int dys = npx + 4;                     // row stride of the dY band: keeps rows 16-byte aligned, spreads banks
+    const int dys = STAGING == 1 ? npx : npx + 4;   // row stride of the dY band (TMA writes dense rows)
     const int win_h = (pl.bp - 1) * g.stride_h + R, win_w = (pl.bq - 1) * g.stride_w + S;
-    const int stage_floats = TK * dys + win_h * win_w * TC;   // a multiple of four
-    // two stages: the next item is fetched while the current one is consumed
+    const int stage_floats = (TK * dys + win_h * win_w * TC + 31) & ~31;   // stages start 128-byte aligned
 
     const int tile = blockIdx.x, split = blockIdx.y;
     const int k0 = (tile / pl.tiles_c) * TK, c0 = (tile % pl.tiles_c) * TC;
@@ -144,21 +133,47 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
 
     const int per = (pl.items + pl.splits - 1) / pl.splits;
     const int it_begin = split * per, it_end = min(pl.items, (split + 1) * per);
-    if (it_begin < it_end) {
-        stage_item<T, ASYNC, TK, TC>(x, dy, smem, smem + TK * dys, g, pl, it_begin, k0, c0, dys, win_h, win_w);
-        if (ASYNC) cp_async_commit();
+    const uint32_t tx_bytes = (uint32_t)(TK * npx + win_h * win_w * TC) * 4u;
+    auto tma_issue = [&](int it, int stage) {     // one thread: both boxes of item `it` into `stage`
+        const int n = it / (pl.bands_p * pl.bands_q);
+        const int band = it % (pl.bands_p * pl.bands_q);
+        const int p0 = (band / pl.bands_q) * pl.bp;
+        const uint32_t full = smem_u32(&bar_full[stage]);
+        const uint32_t dst = smem_u32(smem + stage * stage_floats);
+        mbar_expect_tx(full, tx_bytes);
+        tma_load_3d(dst, &map_dy, full, p0 * g.q, k0, n);
+        tma_load_4d(dst + TK * npx * 4, &map_x, full, c0, -g.pad_w, p0 * g.stride_h - g.pad_h, n);
+    };
+    if (STAGING == 1) {
+        if (threadIdx.x == 0) {
+            s_fail = 0;
+            mbar_init(smem_u32(&bar_full[0]), 1); mbar_init(smem_u32(&bar_full[1]), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && it_begin < it_end) tma_issue(it_begin, 0);
+    } else if (it_begin < it_end) {
+        stage_item<T, false, TK, TC>(x, dy, smem, smem + TK * dys, g, pl, it_begin, k0, c0, dys, win_h, win_w);
     }
     int stage = 0;
+    uint32_t phase[2] = {0u, 0u};
     for (int it = it_begin; it < it_end; ++it, stage ^= 1) {
         float* cur = smem + stage * stage_floats;
         if (it + 1 < it_end) {
-            float* nxt = smem + (stage ^ 1) * stage_floats;
-            stage_item<T, ASYNC, TK, TC>(x, dy, nxt, nxt + TK * dys, g, pl, it + 1, k0, c0, dys, win_h, win_w);
-            if (ASYNC) { cp_async_commit(); cp_async_wait<1>(); }
-        } else if (ASYNC) {
-            cp_async_wait<0>();
+            if (STAGING == 1) { if (threadIdx.x == 0) tma_issue(it + 1, stage ^ 1); }
+            else {
+                float* nxt = smem + (stage ^ 1) * stage_floats;
+                stage_item<T, false, TK, TC>(x, dy, nxt, nxt + TK * dys, g, pl, it + 1, k0, c0, dys, win_h, win_w);
+            }
         }
-        __syncthreads();
+        if (STAGING == 1) {
+            if (!mbar_wait(smem_u32(&bar_full[stage]), phase[stage])) s_fail = 1;   // bounded wait gave up
+            phase[stage] ^= 1u;
+            __syncthreads();
+            if (s_fail) { if (threadIdx.x == 0) atomicOr(status, 1u); break; }       // uniform exit
+        } else {
+            __syncthreads();
+        }
         const float* s_dy = cur + otk * TKT * dys;
         const float* s_x = cur + TK * dys + otc * TCT;
         int pp = pg / pl.bq, qq = pg % pl.bq;
@@ -250,8 +265,8 @@ direct_element_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* 
     dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * acc;
 }
 
-template <typename T> constexpr bool kAsyncOk = false;      // cp.async staging copies raw fp32
-template <> constexpr bool kAsyncOk<float> = true;
+template <typename T> constexpr bool kTmaOk = false;      // TMA staging copies raw fp32
+template <> constexpr bool kTmaOk<float> = true;
 
 // thread-tile shape of each variant
 struct Variant { int tkt, tct, otk, otc; };
@@ -265,15 +280,15 @@ Variant variant_for(const Geom& g)
 size_t smem_for(const Geom& g, const Variant& v, int bp, int bq)
 {
     const int tk = v.tkt * v.otk, tc = v.tct * v.otc, ot = v.otk * v.otc;
-    const size_t stage = 2 * sizeof(float) * ((size_t)tk * (bp * bq + 4) + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * tc);
+    const size_t stage = 2 * sizeof(float) * ((((size_t)tk * (bp * bq + 4) + (size_t)((bp - 1) * g.stride_h + g.r) * ((bq - 1) * g.stride_w + g.s) * tc) + 31) & ~(size_t)31);
     const int sets = ot >= 32 ? kThreads / ot : kThreads / 32;
     const size_t red = sizeof(float) * (size_t)sets * ot * 16;
     return stage > red ? stage : red;
 }
 
 template <typename T>
-cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, const Geom& g, const DirectPlan& pl,
-                     cudaStream_t stream)
+cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_t* status, const Geom& g,
+                     const DirectPlan& pl, cudaStream_t stream)
 {
     if (!pl.tiled) {
         const long long total = (long long)g.k * g.r * g.s * g.c;
@@ -282,19 +297,39 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, const G
         return cudaGetLastError();
     }
     const Variant v = variant_for(g);
+    const int tk = v.tkt * v.otk, tc = v.tct * v.otc;
     const size_t smem = smem_for(g, v, pl.bp, pl.bq);
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
-    const bool use_async = kAsyncOk<T> && pl.vec_dy && pl.vec_x;
+    const int npx = pl.bp * pl.bq, pq = g.p * g.q;
+    const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
+    // TMA staging: fp32 tiles copied as they are
+    bool use_tma = kTmaOk<T> && pl.vec_dy && pl.vec_x && pq % 4 == 0 && npx <= 256 && win_w <= 256 && win_h <= 256 &&
+                   encode_fn() != nullptr;
+    CUtensorMap map_dy{}, map_x{};
+    if (use_tma) {
+        cuuint64_t d3[3] = {(cuuint64_t)pq, (cuuint64_t)g.k, (cuuint64_t)g.n};
+        cuuint64_t s3[2] = {(cuuint64_t)pq * 4, (cuuint64_t)g.k * pq * 4};
+        cuuint32_t b3[3] = {(cuuint32_t)npx, (cuuint32_t)tk, 1}, e3[3] = {1, 1, 1};
+        cuuint64_t d4[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
+        cuuint64_t s4[3] = {(cuuint64_t)g.c * 4, (cuuint64_t)g.w * g.c * 4, (cuuint64_t)g.h * g.w * g.c * 4};
+        cuuint32_t b4[4] = {(cuuint32_t)tc, (cuuint32_t)win_w, (cuuint32_t)win_h, 1}, e4[4] = {1, 1, 1, 1};
+        if (encode_fn()(&map_dy, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<T*>(dy), d3, s3, b3, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            encode_fn()(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<T*>(x), d4, s4, b4, e4, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            use_tma = false;
+    }
     bool done = false;
+#define GACONV_DIRECT_LAUNCH(ST, RR, A, B, C, D)                                                                                 \
+    {                                                                                                                            \
+        auto kern = direct_tiled_kernel<T, ST, RR, RR, A, B, C, D>;                                                              \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                \
+        kern<<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, status, map_dy, map_x, g, pl);                                \
+    }
 #define GACONV_DIRECT_CASE(RR, A, B, C, D)                                                                     \
     if (!done && g.r == RR && v.tkt == A && v.tct == B && v.otk == C && v.otc == D) {                          \
-        if (use_async) {                                                                                       \
-            if (smem > 48 * 1024) cudaFuncSetAttribute(direct_tiled_kernel<T, kAsyncOk<T>, RR, RR, A, B, C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-            direct_tiled_kernel<T, kAsyncOk<T>, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
-        } else {                                                                                               \
-            if (smem > 48 * 1024) cudaFuncSetAttribute(direct_tiled_kernel<T, false, RR, RR, A, B, C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-            direct_tiled_kernel<T, false, RR, RR, A, B, C, D><<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, g, pl); \
-        }                                                                                                      \
+        if (use_tma) GACONV_DIRECT_LAUNCH(kTmaOk<T> ? 1 : 0, RR, A, B, C, D)                                   \
+        else GACONV_DIRECT_LAUNCH(0, RR, A, B, C, D)                                                           \
         done = true;                                                                                           \
     }
     GACONV_DIRECT_CASE(1, 4, 4, 4, 4)
@@ -304,6 +339,7 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, const G
     GACONV_DIRECT_CASE(5, 2, 2, 8, 8)
     GACONV_DIRECT_CASE(5, 1, 4, 16, 1)
 #undef GACONV_DIRECT_CASE
+#undef GACONV_DIRECT_LAUNCH
     if (!done) return cudaErrorInvalidValue;
     note_launch();
     cudaError_t e = cudaGetLastError();
@@ -351,13 +387,12 @@ DirectPlan plan_direct(const Geom& g)
     return pl;
 }
 
-cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
+cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* status,
                           const Geom& g, const DirectPlan& plan, cudaStream_t stream)
 {
-    (void)counters;
     if (g.bf16)
-        return launch_t(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy), dw, partial, g, plan, stream);
-    return launch_t(static_cast<const float*>(x), static_cast<const float*>(dy), dw, partial, g, plan, stream);
+        return launch_t(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy), dw, partial, status, g, plan, stream);
+    return launch_t(static_cast<const float*>(x), static_cast<const float*>(dy), dw, partial, status, g, plan, stream);
 }
 
 }  // namespace gaconv

@@ -66,14 +66,23 @@ random_kernel(float* __restrict__ dw, size_t count, Geom g, uint32_t key0, uint3
         reinterpret_cast<float4*>(dw)[j] = make_float4(std * z[0], std * z[1], std * z[2], std * z[3]);
         return;
     }
-    for (int t = 0; t < 4; ++t) {
-        const size_t i = 4 * j + t;
-        if (i >= count) break;
-        // logical [k][c][r][s] position of element i -> offset in the chosen dW layout
-        const int s = (int)(i % g.s); size_t rest = i / g.s;
-        const int r = (int)(rest % g.r); rest /= g.r;
-        const int cc = (int)(rest % g.c); const int k = (int)(rest / g.c);
+    // logical [k][c][r][s] position of element 4j, decoded once (32-bit arithmetic when it fits), then
+    // stepped; each element goes to its offset in the chosen dW layout
+    int s, r, cc, k;
+    if (count < (1ull << 31)) {
+        uint32_t rest = (uint32_t)(4 * j);
+        s = rest % (uint32_t)g.s; rest /= (uint32_t)g.s;
+        r = rest % (uint32_t)g.r; rest /= (uint32_t)g.r;
+        cc = rest % (uint32_t)g.c; k = rest / (uint32_t)g.c;
+    } else {
+        size_t rest = 4 * j;
+        s = (int)(rest % g.s); rest /= g.s;
+        r = (int)(rest % g.r); rest /= g.r;
+        cc = (int)(rest % g.c); k = (int)(rest / g.c);
+    }
+    for (int t = 0; t < 4 && 4 * j + t < count; ++t) {
         dw[k * g.ws_k + cc * g.ws_c + r * g.ws_r + s * g.ws_s] = std * z[t];
+        if (++s == g.s) { s = 0; if (++r == g.r) { r = 0; if (++cc == g.c) { cc = 0; ++k; } } }
     }
 }
 

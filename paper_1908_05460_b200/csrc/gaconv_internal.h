@@ -68,7 +68,7 @@ struct DirectPlan {
     bool vec_dy, vec_x;     // 4-element vector loads usable for the dY band / the X window
 };
 DirectPlan plan_direct(const Geom& g);
-cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters,
+cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* status,
                           const Geom& g, const DirectPlan& plan, cudaStream_t stream);
 
 // ---- exact filter gradient on tcgen05 tensor cores (bf16, NHWC X, shapes its tiling covers) ----

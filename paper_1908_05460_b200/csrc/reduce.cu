@@ -1,8 +1,8 @@
 // Fixed-order sum of split partial results:  dw[i] = alpha * sum_{sp} partial[sp][i], i < count.
 // partial is [splits][count] in the element order of dw.  A block handles 32 columns (float4 columns
-// when count is a multiple of four); each of its 32 warps sums an interleaved subset of the splits in
-// ascending order, and warp 0 adds the 32 subtotals in warp order, so the result does not depend
-// on scheduling.
+// when count is a multiple of four); each of its W warps (W = splits rounded up to a power of two, at
+// most 32) sums an interleaved subset of the splits in ascending order, and warp 0 adds the W
+// subtotals in warp order, so the result does not depend on scheduling.
 #include "gaconv_internal.h"
 
 namespace gaconv {
@@ -23,19 +23,19 @@ __global__ void __launch_bounds__(32 * kReduceWarps)
 reduce_splits_kernel(const V* __restrict__ partial, V* __restrict__ dw, size_t count, int splits, float alpha)
 {
     __shared__ V sm[kReduceWarps][32];
-    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + lane;
     V acc = vzero<V>();
     if (i < count) {
         const V* p = partial + i;
 #pragma unroll 5
-        for (int sp = grp; sp < splits; sp += kReduceWarps) vadd(acc, __ldcg(p + (size_t)sp * count));
+        for (int sp = grp; sp < splits; sp += warps) vadd(acc, __ldcg(p + (size_t)sp * count));
     }
     sm[grp][lane] = acc;
     __syncthreads();
     if (grp == 0 && i < count) {
         V t = sm[0][lane];
-        const int used = splits < kReduceWarps ? splits : kReduceWarps;
+        const int used = splits < warps ? splits : warps;
         for (int w = 1; w < used; ++w) vadd(t, sm[w][lane]);
         dw[i] = vscale(t, alpha);
     }
@@ -45,12 +45,15 @@ reduce_splits_kernel(const V* __restrict__ partial, V* __restrict__ dw, size_t c
 
 cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int splits, float alpha, cudaStream_t stream)
 {
+    // as many warps per block as there are splits to share out (a power of two, at most 32)
+    int warps = 1;
+    while (warps < splits && warps < kReduceWarps) warps *= 2;
     if (count % 4 == 0) {
         const size_t c4 = count / 4;
-        reduce_splits_kernel<float4><<<(unsigned)((c4 + 31) / 32), 32 * kReduceWarps, 0, stream>>>(
+        reduce_splits_kernel<float4><<<(unsigned)((c4 + 31) / 32), 32 * warps, 0, stream>>>(
             reinterpret_cast<const float4*>(partial), reinterpret_cast<float4*>(dw), c4, splits, alpha);
     } else {
-        reduce_splits_kernel<float><<<(unsigned)((count + 31) / 32), 32 * kReduceWarps, 0, stream>>>(partial, dw, count, splits, alpha);
+        reduce_splits_kernel<float><<<(unsigned)((count + 31) / 32), 32 * warps, 0, stream>>>(partial, dw, count, splits, alpha);
     }
     note_launch();
     return cudaGetLastError();

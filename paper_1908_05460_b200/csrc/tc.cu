@@ -27,49 +27,11 @@
 #include <cstring>
 
 #include "gaconv_internal.h"
+#include "tma.cuh"
 
 namespace gaconv {
 namespace {
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the limit expires.
-constexpr uint32_t kWaitLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// Same bound in wall time, but the warp sleeps between polls so that it does not take issue slots
-// from the producer and MMA threads while the main loop runs.
-__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(128);
-    }
-    return false;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
@@ -108,6 +70,8 @@ struct TcParams {
     int stage_bytes, stages;
     int ksteps;         // ci*bp*Q/16
     int tmem_cols;      // power of two >= 32
+    int rsplit;         // 1: a CTA handles ONE filter row (tile index carries r); M = 128, N = s * 64
+    int rc;             // filter rows per CTA: g.r, or 1 when rsplit
     int issuers;        // MMA-issuing warps: min(R, 3); issuer i takes filter rows i, i+issuers, ...
     uint32_t idesc;
     int timeline;       // 1: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
@@ -133,7 +97,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const Geom& g = P.g;
 
     const int tile = blockIdx.x, split = blockIdx.y;
-    const int k0 = (tile / P.tiles_c) * P.m, c0 = (tile % P.tiles_c) * P.ct;
+    const int r_lo = P.rsplit ? tile % g.r : 0;                 // first filter row of this CTA
+    const int kc_tile = P.rsplit ? tile / g.r : tile;
+    const int k0 = (kc_tile / P.tiles_c) * P.m, c0 = (kc_tile % P.tiles_c) * P.ct;
     const int per = (P.chunks + P.splits - 1) / P.splits;
     const int ch_begin = min(P.chunks, split * per), ch_end = min(P.chunks, ch_begin + per);
     const int nchunks = ch_end - ch_begin;
@@ -182,7 +148,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             if (P.halo) {
                 for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride) tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 - g.pad_h, n0);
             } else {
-                for (int r = 0; r < g.r; ++r)
+                for (int r = r_lo; r < r_lo + P.rc; ++r)
                     for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride)
                         tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 * g.stride_h + r - g.pad_h, n0);
             }
@@ -205,7 +171,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const int ks_per_sub = P.a_sub_px / 16;
         const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4, b_k_step = (16 * b_row_bytes) >> 4;
         const uint32_t b_r_step = (P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
-        const int R = R_T ? R_T : g.r;
+        const int R = R_T ? R_T : P.rc;
         const int KS = KS_T ? KS_T : ks_per_sub;
         // this issuer's filter rows: TMEM address of the accumulator and descriptor offset of the row
         constexpr int RI = R_T == 0 ? 3 : (R_T + 2) / 3;           // rows per issuer, at most (R <= 7 -> 3)
@@ -261,13 +227,13 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             const int sp = warp & 3;
             float* out = P.splits == 1 ? dw : partial + (size_t)split * g.k * g.r * g.s * g.c;
             const float scale = nchunks > 0 ? (P.splits == 1 ? g.alpha : 1.0f) : 0.0f;
-            const int groups = P.m == 128 ? g.r : (g.r + 1) / 2;
+            const int groups = P.m == 128 ? P.rc : (P.rc + 1) / 2;
             const int k = k0 + (P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15));
             const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
             for (int gi = 0; gi < groups; ++gi) {
-                const int r = P.m == 128 ? gi : 2 * gi + (lane >> 4);
-                const bool row_ok = r < g.r && k < g.k;
-                float* row = out + k * g.ws_k + r * g.ws_r;
+                const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's rows
+                const bool row_ok = rl < P.rc && k < g.k;
+                float* row = out + k * g.ws_k + (r_lo + rl) * g.ws_r;
                 const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
                 for (int s = 0; s < g.s; ++s) {
                     float* ps = row + s * g.ws_s;
@@ -314,21 +280,6 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
 CUtensorMapSwizzle swizzle_for(int bytes) {
     return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
 }
@@ -346,7 +297,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     const int pq = g.p * g.q;
     if (pq % 16 != 0 || (pq < 64 && pq != 16 && pq != 32) || (pq >= 64 && pq % 64 != 0)) return false;
     const bool small_map = pq < 64;
-    const bool halo = !small_map && g.stride_h == 1 && g.q % 8 == 0 && 64 % g.q == 0;
+    bool halo = !small_map && g.stride_h == 1 && g.q % 8 == 0 && 64 % g.q == 0;
     if (!small_map && !(g.q <= 64 && 64 % g.q == 0)) return false;        // a 64-pixel box must be whole rows
     if (g.r > 7 || g.s > 7) return false;
 
@@ -356,22 +307,27 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // rows, the fast MN-major format) hold all three filter rows; M = 128 with 32-channel tiles measured
     // about twice slower per FLOP, so it is used only where the tile is narrow anyway.
     P.m = (g.k <= 64 || g.c >= 64) ? 64 : 128;
+    // Many output channels and wide inputs: one filter row per CTA, so that a full-rate M = 128 MMA with a
+    // 64-channel (128-byte row) B tile fits tensor memory (S*64 columns) and the epilogue block shrinks.
+    P.rsplit = (g.k >= 128 && g.c >= 64 && g.r > 1 && env_int("GACONV_TC_RSPLIT", 1)) ? 1 : 0;
+    P.rc = P.rsplit ? 1 : g.r;
+    if (P.rsplit) P.m = 128;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     // channels per tile: one swizzle span wide (16, 32 or 64 channels), limited by MMA N <= 256 and TMEM columns
     int ct = g.c >= 64 ? 64 : g.c >= 32 ? 32 : 16;
-    auto cols_for = [&](int c) { return (P.m == 128 ? g.r : (g.r + 1) / 2) * g.s * c; };
+    auto cols_for = [&](int c) { return (P.m == 128 ? P.rc : (P.rc + 1) / 2) * g.s * c; };
     while (ct > 16 && (g.s * ct > 256 || cols_for(ct) > 512)) ct /= 2;
     if (g.s * ct > 256 || cols_for(ct) > 512) return false;
     if ((g.s * ct) % (P.m == 128 ? 16 : 8) != 0) return false;
     P.ct = ct;
     P.tiles_k = (g.k + P.m - 1) / P.m;
     P.tiles_c = (g.c + ct - 1) / ct;
-    if (P.tiles_k * P.tiles_c > kWsNumCounters) return false;
+    if (P.rsplit) halo = false;          // a single row needs no halo rows: its S tiles are loaded directly
     P.halo = halo ? 1 : 0;
     P.a_sub_px = small_map ? pq : 64;
     P.a_swz = swz_code(P.a_sub_px * 2);
     P.b_swz = swz_code(ct * 2);
-    P.b_tiles = halo ? g.s : g.r * g.s;
+    P.b_tiles = halo ? g.s : P.rc * g.s;
 
     // chunk size: as many rows (or images) as fit a ~48 KiB stage
     const int budget = env_int("GACONV_TC_STAGE_KB", 48) * 1024;
@@ -404,21 +360,22 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.stages = smem_budget / P.stage_bytes;
     if (P.stages > kMaxStages) P.stages = kMaxStages;
     if (P.stages < 2) return false;
-    P.issuers = g.r < 3 ? g.r : 3;
+    P.issuers = P.rc < 3 ? P.rc : 3;
     P.tmem_cols = pow2_ceil(cols_for(ct));
     if (P.tmem_cols > 512) return false;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
     P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
-    const int tiles = P.tiles_k * P.tiles_c;
+    const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
     int splits = env_int("GACONV_TC_SPLITS", 0);
     if (splits <= 0) {
         splits = 148 / tiles;
         if (splits < 1) splits = 1;
-        // partial blocks are written and read back: keep them well below the input bytes
+        // every SM should work; the partial blocks are written and read back (mostly in L2), so cap them
+        // only where they would dwarf the inputs
         const size_t out_bytes = (size_t)g.k * g.r * g.s * g.c * 4;
         const size_t in_bytes = ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 2;
-        while (splits > 1 && (size_t)splits * out_bytes > in_bytes / 2 + (1 << 20)) --splits;
+        while (splits > 1 && (size_t)splits * out_bytes > 4 * in_bytes + (8u << 20)) --splits;
     }
     if (splits > P.chunks) splits = P.chunks;
     {   // no empty splits: every CTA gets ceil(chunks / splits) chunks except possibly the last
@@ -467,11 +424,11 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     // dynamic shared memory: stages, 1 KiB of alignment slack, and a tail so that the MMA's read of
     // all M rows of an A box with fewer valid rows stays inside the allocation
     const size_t smem = (size_t)P.stages * P.stage_bytes + 1024 + (size_t)P.m * 128;
-    dim3 grid(P.tiles_k * P.tiles_c, P.splits);
+    dim3 grid(P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1), P.splits);
     const int ks = P.a_sub_px / 16;
     cudaError_t err = cudaErrorInvalidValue;
 #define GACONV_TC_CASE(RR, KK)                                                                                     \
-    if (err == cudaErrorInvalidValue && (RR == 0 || (g.r == RR && ks == KK))) {                                     \
+    if (err == cudaErrorInvalidValue && (RR == 0 || (P.rc == RR && ks == KK))) {                                     \
         static size_t configured = 0;                                                                              \
         err = cudaSuccess;                                                                                         \
         if (smem > configured) {                                                                                   \
