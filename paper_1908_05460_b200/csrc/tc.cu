@@ -64,7 +64,9 @@ struct TcParams {
     int a_sub_bytes;    // kb * a_sub_px * 2
     int a_region_bytes; // a_subs * a_sub_bytes rounded up to 1 KiB (B tiles start there)
     int a_swz, b_swz;   // swizzle codes of the descriptors
-    int b_tiles;        // S (halo) or R*S
+    int b_tiles;        // S (halo) or R*S; 1 when wide
+    int wide;           // 1: ONE tile of (rows + rc - 1) x (Q + S - 1) pixels; a column shift is a one-pixel
+                        //    descriptor offset (leading byte offset = one pixel row), a row shift a whole tile row
     int b_tile_stride;  // bytes between consecutive B tiles (multiple of 1024)
     int b_tile_bytes;   // bytes one TMA writes per B tile
     int stage_bytes, stages;
@@ -145,7 +147,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                 int px = p0 * g.q;
                 for (int b = 0; b < P.a_subs; ++b, px += 64) tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, px, k0, n0);
             }
-            if (P.halo) {
+            if (P.wide) {
+                tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
+            } else if (P.halo) {
                 for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride) tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 - g.pad_h, n0);
             } else {
                 for (int r = r_lo; r < r_lo + P.rc; ++r)
@@ -166,11 +170,20 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         // descriptors are assembled from a constant high word and a low word that only advances
         const uint32_t a_row_bytes = P.a_sub_px * 2, b_row_bytes = P.ct * 2;
         const uint32_t a_hi = ((8 * a_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.a_swz << 29);
-        const uint32_t b_hi = ((8 * b_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
-        const uint32_t a_lo_c = 1u << 16, b_lo_c = (((uint32_t)P.b_tile_stride >> 4) & 0x3fffu) << 16;
+        const uint32_t wt = g.q + g.s - 1;                       // pixels per tile row in wide mode
+        // stride between the two 8-pixel halves of a k-step: contiguous, except in wide mode when a k-step spans two rows
+        const uint32_t b_sbo = (P.wide && g.q == 8) ? wt * b_row_bytes : 8 * b_row_bytes;
+        const uint32_t b_hi = (b_sbo >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
+        const uint32_t a_lo_c = 1u << 16, b_lo_c = (((P.wide ? b_row_bytes : (uint32_t)P.b_tile_stride) >> 4) & 0x3fffu) << 16;
         const int ks_per_sub = P.a_sub_px / 16;
-        const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4, b_k_step = (16 * b_row_bytes) >> 4;
-        const uint32_t b_r_step = (P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
+        const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4;
+        const uint32_t b_r_step = (P.wide ? wt * b_row_bytes : P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
+        // descriptor offset of k-step k4 inside an A box, and the advance from one A box to the next
+        uint32_t b_k_off[4];
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+            b_k_off[k4] = (P.wide ? (((16u * k4) / g.q) * wt + (16u * k4) % g.q) * b_row_bytes : 16u * k4 * b_row_bytes) >> 4;
+        const uint32_t b_sub_step = (P.wide ? (uint32_t)(P.a_sub_px / g.q) * wt * b_row_bytes : (uint32_t)P.a_sub_px * b_row_bytes) >> 4;
         const int R = R_T ? R_T : P.rc;
         const int KS = KS_T ? KS_T : ks_per_sub;
         // this issuer's filter rows: TMEM address of the accumulator and descriptor offset of the row
@@ -206,11 +219,11 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                     if (!(fresh && k4 == 0)) {
 #pragma unroll
                         for (int i = 0; i < RI; ++i)
-                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + 2 * k4), b_hi64 | (b_lo + k4 * b_k_step + b_row[i]), idesc);
+                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + 2 * k4), b_hi64 | (b_lo + b_k_off[k4] + b_row[i]), idesc);
                     }
                 }
                 fresh = false;
-                b_lo += KS * b_k_step;
+                b_lo += b_sub_step;
             }
             umma_commit(smem_u32(&bar_empty[st]));   // frees the stage once these MMAs have read it
             if (++st == P.stages) { st = 0; ph ^= 1; }
@@ -327,7 +340,9 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.a_sub_px = small_map ? pq : 64;
     P.a_swz = swz_code(P.a_sub_px * 2);
     P.b_swz = swz_code(ct * 2);
-    P.b_tiles = halo ? g.s : P.rc * g.s;
+    // wide tile: stride 1, whole rows per chunk, k-steps inside a row (Q a multiple of 16) or exactly two rows (Q = 8)
+    P.wide = (env_int("GACONV_TC_WIDE", 1) && !small_map && g.stride_h == 1 && (g.q % 16 == 0 || g.q == 8) && 64 % g.q == 0) ? 1 : 0;
+    P.b_tiles = P.wide ? 1 : halo ? g.s : P.rc * g.s;
 
     // chunk size: as many rows (or images) as fit a ~48 KiB stage
     const int budget = env_int("GACONV_TC_STAGE_KB", 48) * 1024;
@@ -335,8 +350,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
         const int px = ci * bp * g.q;
         *a_subs = small_map ? ci : px / 64;
         const int a_bytes = ((small_map ? P.kb * pq * 2 * ci : *a_subs * P.kb * 128) + 1023) / 1024 * 1024;
-        const int rows = halo ? bp + g.r - 1 : bp;
-        *tile_bytes = ci * rows * g.q * ct * 2;
+        const int rows = (halo || P.wide) ? bp + P.rc - 1 : bp;
+        *tile_bytes = ci * rows * (P.wide ? g.q + g.s - 1 : g.q) * ct * 2;
         *tile_stride = (*tile_bytes + 1023) / 1024 * 1024;
         return a_bytes + P.b_tiles * *tile_stride;
     };
@@ -414,8 +429,9 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     {   // X as (c, w, h, n), bf16; a box is ct channels x q columns x rows x ci images, stepping by the conv stride
         cuuint64_t dims[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
         cuuint64_t strides[3] = {(cuuint64_t)g.c * 2, (cuuint64_t)g.w * g.c * 2, (cuuint64_t)g.h * g.w * g.c * 2};
-        const int rows = P.halo ? P.bp + g.r - 1 : P.bp;
-        cuuint32_t box[4] = {(cuuint32_t)P.ct, (cuuint32_t)(g.q * g.stride_w), (cuuint32_t)(rows * g.stride_h), (cuuint32_t)P.ci};
+        const int rows = (P.halo || P.wide) ? P.bp + P.rc - 1 : P.bp;
+        const int cols = P.wide ? g.q + g.s - 1 : g.q * g.stride_w;
+        cuuint32_t box[4] = {(cuuint32_t)P.ct, (cuuint32_t)cols, (cuuint32_t)(rows * g.stride_h), (cuuint32_t)P.ci};
         cuuint32_t es[4] = {1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
         if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(P.ct * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
