@@ -50,16 +50,30 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     return GACONV_OK;
 }
 
-struct Top1Layout { size_t idx_off, sum_off, partial_off, total; GatherPlan gp; };
+// Small maps with many channels: the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes) cost more
+// than the dense contraction on tensor cores, and with few pixels per map the sparse tensor is not
+// that sparse (1 - 1/(PQ), Section 2.3).  Then the method is run literally as the paper states it:
+// build the sparse version of dY (one entry per map, the signed sum) and take its exact filter
+// gradient with the tensor-core kernel.
+bool top1_dense_route(const Geom& g, TcPlan* tp)
+{
+    return g.bf16 && g.p * g.q <= 64 && g.c >= 128 && plan_tc(g, tp);
+}
+
+struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, total; GatherPlan gp; TcPlan tp; bool dense; };
 Top1Layout top1_layout(const Geom& g)
 {
     Top1Layout L;
     L.gp = plan_gather(g);
+    L.dense = top1_dense_route(g, &L.tp);
     const size_t maps = (size_t)g.n * g.k;
     L.idx_off = kWsDataOffset;
     L.sum_off = align_up(L.idx_off + maps * sizeof(int32_t), 256);
     L.partial_off = align_up(L.sum_off + maps * sizeof(float), 256);
-    L.total = align_up(L.partial_off + L.gp.partial_bytes, 256);
+    size_t partial = L.gp.partial_bytes;
+    if (L.dense && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
+    L.sparse_off = align_up(L.partial_off + partial, 256);
+    L.total = align_up(L.sparse_off + (L.dense ? maps * g.p * g.q * 2 : 0), 256);
     return L;
 }
 
@@ -189,11 +203,18 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     const Top1Layout L = top1_layout(g);
     st = check_ws(desc, L.total);       // required by every route, so that behaviour does not depend on the kernel picked
     if (st != GACONV_OK) return st;
-    if (top1_fused_supported(g) && desc->algo != GACONV_ALGO_DIRECT)
-        return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     char* ws = static_cast<char*>(desc->workspace);
     int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx_off);
     float* sum = reinterpret_cast<float*>(ws + L.sum_off);
+    if (L.dense && desc->algo != GACONV_ALGO_DIRECT) {
+        void* sparse = ws + L.sparse_off;
+        if (launch_select(dy, idx, sum, sparse, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        return launch_tc(x, sparse, dw, reinterpret_cast<float*>(ws + L.partial_off),
+                         reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
+                         cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    }
+    if (top1_fused_supported(g) && desc->algo != GACONV_ALGO_DIRECT)
+        return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     if (launch_select(dy, idx, sum, nullptr, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
     if (launch_gather(x, idx, sum, dw, reinterpret_cast<float*>(ws + L.partial_off),
                       reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, cs) != cudaSuccess)
