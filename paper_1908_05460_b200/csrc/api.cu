@@ -60,7 +60,7 @@ bool top1_dense_route(const Geom& g, TcPlan* tp)
     return g.bf16 && g.p * g.q <= 64 && g.c >= 128 && plan_tc(g, tp);
 }
 
-struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, total; GatherPlan gp; TcPlan tp; bool dense; };
+struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, scratch_off, total; GatherPlan gp; TcPlan tp; bool dense; };
 Top1Layout top1_layout(const Geom& g)
 {
     Top1Layout L;
@@ -73,11 +73,12 @@ Top1Layout top1_layout(const Geom& g)
     size_t partial = L.gp.partial_bytes;
     if (L.dense && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
     L.sparse_off = align_up(L.partial_off + partial, 256);
-    L.total = align_up(L.sparse_off + (L.dense ? maps * g.p * g.q * 2 : 0), 256);
+    L.scratch_off = align_up(L.sparse_off + (L.dense ? maps * g.p * g.q * 2 : 0), 256);
+    L.total = align_up(L.scratch_off + (L.dense ? L.tp.scratch_bytes : 0), 256);
     return L;
 }
 
-struct ExactLayout { size_t partial_off, total; DirectPlan dp; TcPlan tp; bool tc_ok; };
+struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; bool tc_ok; };
 ExactLayout exact_layout(const Geom& g)
 {
     ExactLayout L;
@@ -86,7 +87,8 @@ ExactLayout exact_layout(const Geom& g)
     L.partial_off = kWsDataOffset;
     size_t partial = L.dp.partial_bytes;
     if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
-    L.total = align_up(L.partial_off + partial, 256);
+    L.scratch_off = align_up(L.partial_off + partial, 256);
+    L.total = align_up(L.scratch_off + (L.tc_ok ? L.tp.scratch_bytes : 0), 256);
     return L;
 }
 
@@ -173,9 +175,8 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (st != GACONV_OK) return st;
     char* ws = static_cast<char*>(desc->workspace);
     if (L.tc_ok && desc->algo != GACONV_ALGO_DIRECT) {
-        cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
-                                  reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws),
-                                  L.tp, static_cast<cudaStream_t>(stream));
+        cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
+                                  reinterpret_cast<uint32_t*>(ws), L.tp, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
@@ -209,9 +210,8 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     if (L.dense && desc->algo != GACONV_ALGO_DIRECT) {
         void* sparse = ws + L.sparse_off;
         if (launch_select(dy, idx, sum, sparse, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
-        return launch_tc(x, sparse, dw, reinterpret_cast<float*>(ws + L.partial_off),
-                         reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
-                         cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+        return launch_tc(x, sparse, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
+                         reinterpret_cast<uint32_t*>(ws), L.tp, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     if (top1_fused_supported(g) && desc->algo != GACONV_ALGO_DIRECT)
         return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;

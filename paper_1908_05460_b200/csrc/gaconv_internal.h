@@ -74,10 +74,11 @@ cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* parti
 // ---- exact filter gradient on tcgen05 tensor cores (bf16, NHWC X, shapes its tiling covers) ----
 struct TcPlan {
     size_t partial_bytes;
+    size_t scratch_bytes;                   // extra device scratch (transposed dY for very small maps)
     alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
 };
 bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel
-cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters, uint32_t* status,
+cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* status,
                       const TcPlan& plan, cudaStream_t stream);
 
 }  // namespace gaconv

@@ -65,6 +65,11 @@ struct TcParams {
     int a_region_bytes; // a_subs * a_sub_bytes rounded up to 1 KiB (B tiles start there)
     int a_swz, b_swz;   // swizzle codes of the descriptors
     int b_tiles;        // S (halo) or R*S; 1 when wide
+    int tiny;           // 1: maps of fewer than 16 pixels: A comes from a transposed copy dYt[n][pq][k] (MN-major,
+                        //    64 channels per 128-byte row); chunks are whole images, 16 reduction rows per k-step
+    int by_image;       // 1: a chunk is ci whole images (maps under 64 pixels)
+    int a_k4_step;      // descriptor advance (16-byte units) from one k-step to the next inside an A box
+    int a_lbo;          // leading byte offset of the A descriptor
     int wide;           // 1: ONE tile of (rows + rc - 1) x (Q + S - 1) pixels; a column shift is a one-pixel
                         //    descriptor offset (leading byte offset = one pixel row), a row shift a whole tile row
     int b_tile_stride;  // bytes between consecutive B tiles (multiple of 1024)
@@ -86,8 +91,7 @@ constexpr int kMaxStages = 8;
 template <int R_T, int KS_T>
 __global__ void __launch_bounds__(256, 1)
 exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
-                float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters,
-                uint32_t* __restrict__ status, const TcParams P)
+                float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ status, const TcParams P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc;
@@ -128,11 +132,11 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         // ------------------------------------------------------------------ TMA producer
         // chunk coordinates advance incrementally: no division inside the loop
         int n0, p0;
-        const bool whole_maps = P.a_sub_px < 64;
+        const bool whole_maps = P.by_image != 0;
         const int cpi = whole_maps ? 1 : g.p / P.bp;
         if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
-        const uint32_t tx_bytes = P.a_subs * P.a_sub_bytes + P.b_tiles * P.b_tile_bytes;
+        const uint32_t tx_bytes = (P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes;
         int issued = 0, st = 0, ph = 0;
         for (int it = 0; it < nchunks; ++it) {
             if (it >= P.stages && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1)) { s_abort = 1; atomicOr(status, 1u); break; }
@@ -141,7 +145,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             const uint32_t sa = smem_base + st * P.stage_bytes;
             uint32_t sb = sa + P.a_region_bytes;
             mbar_expect_tx(full, tx_bytes);
-            if (whole_maps) {
+            if (P.tiny) {                                                        // one box per 64-channel atom
+                for (int a = 0; a * 64 < P.m; ++a) tma_load_3d(sa + a * P.a_lbo, &map_dy, full, k0 + 64 * a, 0, n0);
+            } else if (whole_maps) {
                 tma_load_3d(sa, &map_dy, full, 0, k0, n0);                       // ci whole maps in one box
             } else {
                 int px = p0 * g.q;
@@ -168,14 +174,15 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const int issuer = warp - 1;
         // ------------------------------------------------------------------ MMA issuer
         // descriptors are assembled from a constant high word and a low word that only advances
-        const uint32_t a_row_bytes = P.a_sub_px * 2, b_row_bytes = P.ct * 2;
+        const uint32_t a_row_bytes = P.tiny ? 128u : P.a_sub_px * 2, b_row_bytes = P.ct * 2;
         const uint32_t a_hi = ((8 * a_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.a_swz << 29);
         const uint32_t wt = g.q + g.s - 1;                       // pixels per tile row in wide mode
         // stride between the two 8-pixel halves of a k-step: contiguous, except in wide mode when a k-step spans two rows
         const uint32_t b_sbo = (P.wide && g.q == 8) ? wt * b_row_bytes : 8 * b_row_bytes;
         const uint32_t b_hi = (b_sbo >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
-        const uint32_t a_lo_c = 1u << 16, b_lo_c = (((P.wide ? b_row_bytes : (uint32_t)P.b_tile_stride) >> 4) & 0x3fffu) << 16;
+        const uint32_t a_lo_c = (((uint32_t)P.a_lbo >> 4) & 0x3fffu) << 16, b_lo_c = (((P.wide ? b_row_bytes : (uint32_t)P.b_tile_stride) >> 4) & 0x3fffu) << 16;
         const int ks_per_sub = P.a_sub_px / 16;
+        const uint32_t a_k4 = (uint32_t)P.a_k4_step;
         const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4;
         const uint32_t b_r_step = (P.wide ? wt * b_row_bytes : P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
         // descriptor offset of k-step k4 inside an A box, and the advance from one A box to the next
@@ -219,7 +226,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                     if (!(fresh && k4 == 0)) {
 #pragma unroll
                         for (int i = 0; i < RI; ++i)
-                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + 2 * k4), b_hi64 | (b_lo + b_k_off[k4] + b_row[i]), idesc);
+                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + a_k4 * k4), b_hi64 | (b_lo + b_k_off[k4] + b_row[i]), idesc);
                     }
                 }
                 fresh = false;
@@ -292,6 +299,20 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     }
 }
 
+// dYt[n][j][k] = dY[n][k][j] for maps of fewer than 16 pixels (the map is too short for a TMA row).
+__global__ void __launch_bounds__(256)
+transpose_dy_kernel(const __nv_bfloat16* __restrict__ dy, __nv_bfloat16* __restrict__ dyt, int n, int k, int pq)
+{
+    const size_t total = (size_t)n * k * pq;
+    const size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // output index: ((n*pq + j)*k + kk)
+    if (o >= total) return;
+    const int kk = (int)(o % k);
+    const size_t rest = o / k;
+    const int j = (int)(rest % pq);
+    const size_t nn = rest / pq;
+    dyt[o] = dy[(nn * k + kk) * pq + j];
+}
+
 // ---------------------------------------------------------------- host side
 CUtensorMapSwizzle swizzle_for(int bytes) {
     return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
@@ -308,7 +329,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
     if (g.xs_c != 1 || g.c % 8 != 0) return false;                       // NHWC with 16-byte pixel rows
     if (g.stride_h != g.stride_w) return false;
     const int pq = g.p * g.q;
-    if (pq % 16 != 0 || (pq < 64 && pq != 16 && pq != 32) || (pq >= 64 && pq % 64 != 0)) return false;
+    const bool tiny = pq < 16 && 16 % pq == 0 && g.k % 8 == 0 && (size_t)g.n * pq >= 64;
+    if (!tiny && (pq % 16 != 0 || (pq < 64 && pq != 16 && pq != 32) || (pq >= 64 && pq % 64 != 0))) return false;
     const bool small_map = pq < 64;
     bool halo = !small_map && g.stride_h == 1 && g.q % 8 == 0 && 64 % g.q == 0;
     if (!small_map && !(g.q <= 64 && 64 % g.q == 0)) return false;        // a 64-pixel box must be whole rows
@@ -326,6 +348,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.rc = P.rsplit ? 1 : g.r;
     if (P.rsplit) P.m = 128;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
+    P.tiny = tiny ? 1 : 0;
+    P.by_image = small_map ? 1 : 0;
     // channels per tile: one swizzle span wide (16, 32 or 64 channels), limited by MMA N <= 256 and TMEM columns
     int ct = g.c >= 64 ? 64 : g.c >= 32 ? 32 : 16;
     auto cols_for = [&](int c) { return (P.m == 128 ? P.rc : (P.rc + 1) / 2) * g.s * c; };
@@ -337,8 +361,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.tiles_c = (g.c + ct - 1) / ct;
     if (P.rsplit) halo = false;          // a single row needs no halo rows: its S tiles are loaded directly
     P.halo = halo ? 1 : 0;
-    P.a_sub_px = small_map ? pq : 64;
-    P.a_swz = swz_code(P.a_sub_px * 2);
+    P.a_sub_px = tiny ? 64 : small_map ? pq : 64;      // tiny: 64 reduction rows (images x pixels) per A box
+    P.a_swz = swz_code(tiny ? 128 : P.a_sub_px * 2);
     P.b_swz = swz_code(ct * 2);
     // wide tile: stride 1, whole rows per chunk, k-steps inside a row (Q a multiple of 16) or exactly two rows (Q = 8)
     P.wide = (env_int("GACONV_TC_WIDE", 1) && !small_map && g.stride_h == 1 && (g.q % 16 == 0 || g.q == 8) && 64 % g.q == 0) ? 1 : 0;
@@ -348,15 +372,18 @@ bool plan_tc(const Geom& g, TcPlan* out)
     const int budget = env_int("GACONV_TC_STAGE_KB", 48) * 1024;
     auto stage_bytes = [&](int ci, int bp, int* a_subs, int* tile_bytes, int* tile_stride) {
         const int px = ci * bp * g.q;
-        *a_subs = small_map ? ci : px / 64;
-        const int a_bytes = ((small_map ? P.kb * pq * 2 * ci : *a_subs * P.kb * 128) + 1023) / 1024 * 1024;
+        *a_subs = tiny ? px / 64 : small_map ? ci : px / 64;
+        const int a_bytes = ((tiny ? (P.m / 64) * px * 128 : small_map ? P.kb * pq * 2 * ci : *a_subs * P.kb * 128) + 1023) / 1024 * 1024;
         const int rows = (halo || P.wide) ? bp + P.rc - 1 : bp;
         *tile_bytes = ci * rows * (P.wide ? g.q + g.s - 1 : g.q) * ct * 2;
         *tile_stride = (*tile_bytes + 1023) / 1024 * 1024;
         return a_bytes + P.b_tiles * *tile_stride;
     };
     int ci = 1, bp = small_map ? g.p : 64 / g.q, a_subs, tb, ts;
-    if (small_map) {
+    if (tiny) {
+        ci = 64 / pq;                                   // 64 reduction rows = four k-steps per chunk at least
+        while (ci * 2 * pq <= 256 && ci * 2 <= g.n && stage_bytes(ci * 2, bp, &a_subs, &tb, &ts) <= budget) ci *= 2;
+    } else if (small_map) {
         while (ci * 2 <= 16 && ci * 2 <= g.n && stage_bytes(ci * 2, bp, &a_subs, &tb, &ts) <= budget) ci *= 2;
     } else {
         while (bp * 2 <= g.p && g.p % (bp * 2) == 0 && (halo ? bp * 2 + g.r - 1 : bp * 2 * g.stride_h) <= 256 &&
@@ -367,8 +394,10 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.stage_bytes = stage_bytes(ci, bp, &a_subs, &tb, &ts);
     P.stage_bytes = (P.stage_bytes + 1023) / 1024 * 1024;
     P.a_subs = a_subs; P.b_tile_bytes = tb; P.b_tile_stride = ts;
-    P.a_sub_bytes = small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
-    P.a_region_bytes = (P.a_subs * P.a_sub_bytes + 1023) / 1024 * 1024;
+    P.a_sub_bytes = tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
+    P.a_k4_step = tiny ? (16 * 128) >> 4 : 2;
+    P.a_lbo = tiny ? ci * pq * 128 : 16;               // tiny: bytes between the 64-channel atoms of an A tile
+    P.a_region_bytes = ((tiny ? (P.m / 64) * ci * pq * 128 : P.a_subs * P.a_sub_bytes) + 1023) / 1024 * 1024;
     P.ksteps = ci * bp * g.q / 16;
     P.chunks = small_map ? (g.n + ci - 1) / ci : g.n * (g.p / bp);
     const int smem_budget = 200 * 1024;
@@ -379,7 +408,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.tmem_cols = pow2_ceil(cols_for(ct));
     if (P.tmem_cols > 512) return false;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
-    P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
+    P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((tiny ? 1u : 0u) << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
     int splits = env_int("GACONV_TC_SPLITS", 0);
@@ -401,12 +430,13 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.timeline = env_int("GACONV_TC_TIMELINE", 0);
 
     out->partial_bytes = splits > 1 ? (size_t)splits * g.k * g.r * g.s * g.c * 4 : 0;
+    out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
     memcpy(out->opaque, &P, sizeof(P));
     return encode_fn() != nullptr;
 }
 
-cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, uint32_t* counters, uint32_t* status,
+cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* status,
                       const TcPlan& plan, cudaStream_t stream)
 {
     TcParams P;
@@ -417,7 +447,19 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     if (enc == nullptr) return cudaErrorNotSupported;
 
     CUtensorMap map_dy, map_x;
-    {   // dY as (pq, k, n), bf16
+    if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) with 64-channel boxes
+        const size_t total = (size_t)g.n * g.k * pq;
+        transpose_dy_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.n, g.k, pq);
+        note_launch();
+        cuuint64_t dims[3] = {(cuuint64_t)g.k, (cuuint64_t)pq, (cuuint64_t)g.n};
+        cuuint64_t strides[2] = {(cuuint64_t)g.k * 2, (cuuint64_t)g.k * pq * 2};
+        cuuint32_t box[3] = {64, (cuuint32_t)pq, (cuuint32_t)P.ci};
+        cuuint32_t es[3] = {1, 1, 1};
+        if (enc(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, scratch, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    } else {   // dY as (pq, k, n), bf16
         cuuint64_t dims[3] = {(cuuint64_t)pq, (cuuint64_t)g.k, (cuuint64_t)g.n};
         cuuint64_t strides[2] = {(cuuint64_t)pq * 2, (cuuint64_t)g.k * pq * 2};
         cuuint32_t box[3] = {(cuuint32_t)P.a_sub_px, (cuuint32_t)P.kb, (cuuint32_t)(P.a_sub_px < 64 ? P.ci : 1)};
@@ -452,7 +494,7 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
             if (err == cudaSuccess) configured = smem;                                                             \
         }                                                                                                          \
         if (err == cudaSuccess)                                                                                    \
-            exact_tc_kernel<RR, KK><<<grid, 256, smem, stream>>>(map_dy, map_x, dw, partial, counters, status, P);  \
+            exact_tc_kernel<RR, KK><<<grid, 256, smem, stream>>>(map_dy, map_x, dw, partial, status, P);  \
     }
     GACONV_TC_CASE(3, 4)
     GACONV_TC_CASE(3, 1)

@@ -258,6 +258,10 @@ TC_SHAPES = [
     ConvLayer("tc k72", 4, 16, 8, 8, 72, 3, 3, 1, 1),
     ConvLayer("tc 1x1", 4, 32, 16, 16, 48, 1, 1, 1, 0),
     ConvLayer("tc many splits", 128, 16, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("tc 2x2 maps (transposed dY), one row per CTA", 40, 64, 2, 2, 128, 3, 3, 1, 1),
+    ConvLayer("tc 2x2 maps, narrow", 33, 24, 2, 2, 40, 3, 3, 1, 1),
+    ConvLayer("tc 1x1 maps", 70, 32, 1, 1, 64, 1, 1, 1, 0),
+    ConvLayer("tc 128->128@16 one row per CTA", 4, 128, 16, 16, 128, 3, 3, 1, 1),
 ]
 
 
