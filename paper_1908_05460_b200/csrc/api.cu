@@ -176,7 +176,8 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     char* ws = static_cast<char*>(desc->workspace);
     if (L.tc_ok && desc->algo != GACONV_ALGO_DIRECT) {
         cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
-                                  reinterpret_cast<uint32_t*>(ws), L.tp, static_cast<cudaStream_t>(stream));
+                                  reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
+                                  static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),
@@ -211,7 +212,8 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
         void* sparse = ws + L.sparse_off;
         if (launch_select(dy, idx, sum, sparse, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
         return launch_tc(x, sparse, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
-                         reinterpret_cast<uint32_t*>(ws), L.tp, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+                         reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
+                         cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     if (top1_fused_supported(g) && desc->algo != GACONV_ALGO_DIRECT)
         return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;

@@ -78,7 +78,8 @@ struct TcPlan {
     alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
 };
 bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel
-cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* status,
+cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* counters,
+                      uint32_t* status,
                       const TcPlan& plan, cudaStream_t stream);
 
 }  // namespace gaconv

@@ -13,8 +13,9 @@
 //        R-1 halo rows ("halo" mode); otherwise every (r,s) has its own tile ("separate" mode).
 //   D  = R accumulators in tensor memory, fp32.  With M = 64 (K <= 64) an accumulator occupies 16 of
 //        the 32 lanes of each TMEM sub-partition, so two accumulators share the same columns.
-// A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks; the
-// partial blocks of the splits are summed in split order by a second, element-parallel kernel.
+// A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks.  Consecutive
+// splits form a thread-block cluster and add their blocks through distributed shared memory; if a tile
+// has several clusters, a second, element-parallel kernel adds the clusters' slots in order.
 //
 // Warp roles: warp 0 = TMA producer; warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns
 // the TMEM allocation); warps 4..7 = epilogue.  The filter rows are dealt round-robin to the issuers:
@@ -22,6 +23,8 @@
 // Every mbarrier wait is bounded; on expiry the kernel raises the workspace status word, drains
 // the copies it has in flight, frees its tensor memory and returns.
 #include <cuda.h>
+
+#include <cooperative_groups.h>
 
 #include <cstdlib>
 #include <cstring>
@@ -39,6 +42,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc) : "memory");
+}
+// 16 bytes from the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float4 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    return v;
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -65,7 +76,7 @@ struct TcParams {
     int a_region_bytes; // a_subs * a_sub_bytes rounded up to 1 KiB (B tiles start there)
     int a_swz, b_swz;   // swizzle codes of the descriptors
     int b_tiles;        // S (halo) or R*S; 1 when wide
-    int tiny;           // 1: maps of fewer than 16 pixels: A comes from a transposed copy dYt[n][pq][k] (MN-major,
+    int tiny;           // 1: maps of fewer than 64 pixels: A comes from a transposed copy dYt[n][pq][k] (MN-major,
                         //    64 channels per 128-byte row); chunks are whole images, 16 reduction rows per k-step
     int by_image;       // 1: a chunk is ci whole images (maps under 64 pixels)
     int a_k4_step;      // descriptor advance (16-byte units) from one k-step to the next inside an A box
@@ -77,6 +88,7 @@ struct TcParams {
     int stage_bytes, stages;
     int ksteps;         // ci*bp*Q/16
     int tmem_cols;      // power of two >= 32
+    int cl;             // thread-block cluster size along the split dimension (1, 2, 4 or 8); divides splits
     int rsplit;         // 1: a CTA handles ONE filter row (tile index carries r); M = 128, N = s * 64
     int rc;             // filter rows per CTA: g.r, or 1 when rsplit
     int issuers;        // MMA-issuing warps: min(R, 3); issuer i takes filter rows i, i+issuers, ...
@@ -91,7 +103,8 @@ constexpr int kMaxStages = 8;
 template <int R_T, int KS_T>
 __global__ void __launch_bounds__(256, 1)
 exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
-                float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ status, const TcParams P)
+                float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters,
+                uint32_t* __restrict__ status, const TcParams P)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc;
@@ -110,6 +123,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int ch_begin = min(P.chunks, split * per), ch_end = min(P.chunks, ch_begin + per);
     const int nchunks = ch_end - ch_begin;
     const int nmma = g.s * P.ct;
+    float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // reduction block, aliases the stages
+    const int red_stride = P.rc * nmma + 4;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), P.issuers); }
@@ -213,8 +228,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (tl && it == 0 && issuer == 0) tl[1] = clock64();
             const uint32_t sa = smem_base + st * P.stage_bytes;
-            uint32_t a_lo = a_lo_c | (sa >> 4);
-            uint32_t b_lo = b_lo_c | ((sa + P.a_region_bytes) >> 4);
+            // 14-bit start-address fields: in a cluster launch shared addresses carry the CTA rank in high bits
+            uint32_t a_lo = a_lo_c | ((sa >> 4) & 0x3fffu);
+            uint32_t b_lo = b_lo_c | (((sa + P.a_region_bytes) >> 4) & 0x3fffu);
             for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
                 if (fresh) {      // first k-step of this CTA: accumulate flag off
 #pragma unroll
@@ -238,51 +254,39 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         umma_commit(smem_u32(&bar_acc));             // accumulators complete
         if (tl && issuer == 0) tl[2] = clock64();
     } else if (warp >= 4) {
-        // ------------------------------------------------------------------ epilogue: TMEM -> global
+        // ------------------------------------------------------------------ epilogue 1: TMEM -> shared memory
+        // The accumulators go to a [row][column] fp32 block in this CTA's shared memory (the operand
+        // stages are free by now); column = local filter row * nmma + s * ct + c.  Rows are padded by four
+        // floats so that the 32 lanes of a warp, one row each, store 16-byte pieces without bank conflicts.
         const bool ready = mbar_wait_sleepy(smem_u32(&bar_acc), 0);
         if (!ready) { s_abort = 1; atomicOr(status, 1u); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (tl && threadIdx.x == 128) tl[3] = clock64();
         if (ready && !s_abort) {
             const int sp = warp & 3;
-            float* out = P.splits == 1 ? dw : partial + (size_t)split * g.k * g.r * g.s * g.c;
-            const float scale = nchunks > 0 ? (P.splits == 1 ? g.alpha : 1.0f) : 0.0f;
             const int groups = P.m == 128 ? P.rc : (P.rc + 1) / 2;
-            const int k = k0 + (P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15));
-            const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
+            const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
             for (int gi = 0; gi < groups; ++gi) {
-                const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's rows
-                const bool row_ok = rl < P.rc && k < g.k;
-                float* row = out + k * g.ws_k + (r_lo + rl) * g.ws_r;
+                const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's filter rows
+                const bool row_ok = rl < P.rc && k0 + row < g.k;
                 const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
-                for (int s = 0; s < g.s; ++s) {
-                    float* ps = row + s * g.ws_s;
-                    for (int cc = 0; cc < P.ct; cc += 64) {
-                        const uint32_t taddr = tbase + s * P.ct + cc;
-                        // up to four 16-column loads in flight before the single wait
-                        float v[4][16];
-                        const int nld = min(4, (P.ct - cc) >> 4);
+                float* rrow = red + row * red_stride + rl * nmma;
+                for (int col = 0; col < nmma; col += 64) {
+                    float v[4][16];                                        // up to four 16-column loads in flight
+                    const int nld = min(4, (nmma - col) >> 4);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (u < nld) tmem_ld16_nowait(taddr + 16 * u, v[u]);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                        if (!row_ok) continue;
+                    for (int u = 0; u < 4; ++u)
+                        if (u < nld) tmem_ld16_nowait(tbase + col + 16 * u, v[u]);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (!row_ok) continue;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (u >= nld) continue;
-                            const int c = c0 + cc + 16 * u;
-                            if (vec && c + 16 <= g.c) {
-                                float4* p4 = reinterpret_cast<float4*>(ps + c);
+                    for (int u = 0; u < 4; ++u) {
+                        if (u >= nld) continue;
+                        float4* p4 = reinterpret_cast<float4*>(rrow + col + 16 * u);
 #pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4)
-                                    p4[q4] = make_float4(scale * v[u][4 * q4], scale * v[u][4 * q4 + 1],
-                                                         scale * v[u][4 * q4 + 2], scale * v[u][4 * q4 + 3]);
-                            } else {
-#pragma unroll
-                                for (int jj = 0; jj < 16; ++jj)
-                                    if (c + jj < g.c) ps[(c + jj) * g.ws_c] = scale * v[u][jj];
-                            }
-                        }
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            p4[q4] = nchunks > 0 ? make_float4(v[u][4 * q4], v[u][4 * q4 + 1], v[u][4 * q4 + 2], v[u][4 * q4 + 3])
+                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
             }
@@ -290,13 +294,61 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     }
 
     if (tl && threadIdx.x == 128) tl[4] = clock64();
-    // ---------------------------------------------------------------------- teardown
+    // ---------------------------------------------------------------------- TMEM teardown
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(P.tmem_cols) : "memory");
     }
+
+    // ---------------------------------------------------------------------- epilogue 2: split reduction
+    // The cl CTAs of a cluster are consecutive splits of one output tile.  After a cluster barrier CTA
+    // `rank` adds slice `rank` of the block over the cl CTAs through distributed shared memory, in
+    // rank order.  With one cluster per tile the result (times alpha) goes straight to dW; with several,
+    // to the cluster's slot of the partial buffer, which reduce_splits() adds up in slot order afterwards.
+    // A CTA that gave up on a wait still takes part in the barriers, so its peers never wait in vain.
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int cl = P.cl, rank = cl > 1 ? (int)cluster.block_rank() : 0;
+    const int groups_per_tile = P.splits / cl, cgroup = split / cl;
+    if (cl > 1) cluster.sync();
+    const int rows = min(P.m, g.k - k0), cols = P.rc * nmma;
+    const int q_per_row = cols >> 2, quads = rows * q_per_row;
+    const int slice = (quads + cl - 1) / cl;
+    const int f_begin = min(quads, rank * slice), f_end = min(quads, f_begin + slice);
+    const size_t kcrs = (size_t)g.k * g.r * g.s * g.c;
+    const bool direct = groups_per_tile == 1;
+    float* out = direct ? dw : partial + (size_t)cgroup * kcrs;
+    const float scale = direct ? g.alpha : 1.0f;
+    const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
+    auto out_offset = [&](int f, int& c, int& valid) -> size_t {     // quad f -> offset of its first element in dW's layout
+        const int row = f / q_per_row, col = (f - row * q_per_row) << 2;
+        const int rl = col / nmma, sc = col - rl * nmma, s_ = sc / P.ct;
+        c = c0 + sc - s_ * P.ct;
+        valid = max(0, min(4, g.c - c));
+        return (size_t)(k0 + row) * g.ws_k + (size_t)(r_lo + rl) * g.ws_r + (size_t)s_ * g.ws_s + (size_t)c * g.ws_c;
+    };
+    if (!s_abort) {
+        for (int f = f_begin + (int)threadIdx.x; f < f_end; f += blockDim.x) {
+            const int row = f / q_per_row, col = (f - row * q_per_row) << 2;
+            const float* src = red + row * red_stride + col;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int rk = 0; rk < cl; ++rk) {
+                const float4 v = cl > 1 ? ld_dsmem_f4(smem_u32(src), (uint32_t)rk) : *reinterpret_cast<const float4*>(src);
+                t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+            }
+            int c, valid;
+            const size_t off = out_offset(f, c, valid);
+            if (vec && valid == 4) {
+                *reinterpret_cast<float4*>(out + off) = make_float4(scale * t.x, scale * t.y, scale * t.z, scale * t.w);
+            } else {
+                const float tv[4] = {t.x, t.y, t.z, t.w};
+                for (int j = 0; j < valid; ++j) out[off + (size_t)j * g.ws_c] = scale * tv[j];
+            }
+        }
+    }
+    if (cl > 1) cluster.sync();      // peers may still be reading this CTA's block
 }
 
 // dYt[n][j][k] = dY[n][k][j] for maps of fewer than 16 pixels (the map is too short for a TMA row).
@@ -329,7 +381,9 @@ bool plan_tc(const Geom& g, TcPlan* out)
     if (g.xs_c != 1 || g.c % 8 != 0) return false;                       // NHWC with 16-byte pixel rows
     if (g.stride_h != g.stride_w) return false;
     const int pq = g.p * g.q;
-    const bool tiny = pq < 16 && 16 % pq == 0 && g.k % 8 == 0 && (size_t)g.n * pq >= 64;
+    // maps under 64 pixels: K-major rows of dY would be 32 or 64 bytes (or too short for TMA at all) and the
+    // copy engine's cost is per row, so A is taken from a transposed copy with 128-byte rows instead
+    const bool tiny = pq < 64 && 64 % pq == 0 && g.k % 8 == 0 && (size_t)g.n * pq >= 64 && env_int("GACONV_TC_TRANSPOSE_SMALL", 1);
     if (!tiny && (pq % 16 != 0 || (pq < 64 && pq != 16 && pq != 32) || (pq >= 64 && pq % 64 != 0))) return false;
     const bool small_map = pq < 64;
     bool halo = !small_map && g.stride_h == 1 && g.q % 8 == 0 && 64 % g.q == 0;
@@ -410,34 +464,41 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
     P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((tiny ? 1u : 0u) << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
+    // Splits of the reduction: about 128 CTAs in all, in clusters of up to 4 consecutive splits that reduce
+    // through distributed shared memory (clusters of 8 full-SM CTAs measured slower: they are placed GPC by GPC).
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
+    int cl = 1;
+    while (cl * 2 <= 8 && tiles * cl * 2 <= 128 && cl * 2 <= P.chunks) cl *= 2;
+    if (env_int("GACONV_TC_CLUSTER", 4) < cl) cl = env_int("GACONV_TC_CLUSTER", 4) < 1 ? 1 : env_int("GACONV_TC_CLUSTER", 4);
     int splits = env_int("GACONV_TC_SPLITS", 0);
     if (splits <= 0) {
-        splits = 148 / tiles;
+        splits = 128 / tiles;
         if (splits < 1) splits = 1;
-        // every SM should work; the partial blocks are written and read back (mostly in L2), so cap them
-        // only where they would dwarf the inputs
+        // the cluster slots are written and read back (mostly in L2): cap them only where they would dwarf the inputs
         const size_t out_bytes = (size_t)g.k * g.r * g.s * g.c * 4;
         const size_t in_bytes = ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 2;
-        while (splits > 1 && (size_t)splits * out_bytes > 4 * in_bytes + (8u << 20)) --splits;
+        while (splits > cl && (size_t)(splits / cl) * out_bytes > 4 * in_bytes + (8u << 20)) --splits;
     }
     if (splits > P.chunks) splits = P.chunks;
-    {   // no empty splits: every CTA gets ceil(chunks / splits) chunks except possibly the last
-        const int per = (P.chunks + splits - 1) / splits;
-        splits = (P.chunks + per - 1) / per;
-    }
+    splits = splits / cl * cl;                       // whole clusters
+    if (splits < cl) splits = cl;
+    P.cl = cl;
     P.splits = splits;
+    // the reduction block must fit the dynamic shared memory (it reuses the operand stages)
+    const size_t red_bytes = (size_t)P.m * (P.rc * g.s * ct + 4) * 4;
+    if (red_bytes > 212 * 1024) return false;
+    if ((size_t)tiles * cl > kWsNumCounters) return false;
     P.timeline = env_int("GACONV_TC_TIMELINE", 0);
 
-    out->partial_bytes = splits > 1 ? (size_t)splits * g.k * g.r * g.s * g.c * 4 : 0;
+    out->partial_bytes = splits / cl > 1 ? (size_t)(splits / cl) * g.k * g.r * g.s * g.c * 4 : 0;
     out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
     memcpy(out->opaque, &P, sizeof(P));
     return encode_fn() != nullptr;
 }
 
-cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* status,
-                      const TcPlan& plan, cudaStream_t stream)
+cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* counters,
+                      uint32_t* status, const TcPlan& plan, cudaStream_t stream)
 {
     TcParams P;
     memcpy(&P, plan.opaque, sizeof(P));
@@ -481,7 +542,10 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     }
     // dynamic shared memory: stages, 1 KiB of alignment slack, and a tail so that the MMA's read of
     // all M rows of an A box with fewer valid rows stays inside the allocation
-    const size_t smem = (size_t)P.stages * P.stage_bytes + 1024 + (size_t)P.m * 128;
+    size_t smem = (size_t)P.stages * P.stage_bytes;
+    const size_t red_bytes = (size_t)P.m * (P.rc * g.s * P.ct + 4) * 4;
+    if (red_bytes > smem) smem = red_bytes;
+    smem += 1024 + (size_t)P.m * 128;
     dim3 grid(P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1), P.splits);
     const int ks = P.a_sub_px / 16;
     cudaError_t err = cudaErrorInvalidValue;
@@ -493,8 +557,15 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
             err = cudaFuncSetAttribute(exact_tc_kernel<RR, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
             if (err == cudaSuccess) configured = smem;                                                             \
         }                                                                                                          \
-        if (err == cudaSuccess)                                                                                    \
-            exact_tc_kernel<RR, KK><<<grid, 256, smem, stream>>>(map_dy, map_x, dw, partial, status, P);  \
+        if (err == cudaSuccess) {                                                                                  \
+            cudaLaunchConfig_t cfg = {};                                                                           \
+            cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = stream;        \
+            cudaLaunchAttribute attr[1];                                                                           \
+            attr[0].id = cudaLaunchAttributeClusterDimension;                                                      \
+            attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = P.cl; attr[0].val.clusterDim.z = 1;           \
+            cfg.attrs = attr; cfg.numAttrs = 1;                                                                    \
+            err = cudaLaunchKernelEx(&cfg, exact_tc_kernel<RR, KK>, map_dy, map_x, dw, partial, counters, status, P); \
+        }                                                                                                          \
     }
     GACONV_TC_CASE(3, 4)
     GACONV_TC_CASE(3, 1)
@@ -505,7 +576,8 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     if (err != cudaSuccess) return err;
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
-    if (P.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.r * g.s * g.c, P.splits, g.alpha, stream);
+    if (P.splits / P.cl > 1)
+        return reduce_splits(partial, dw, (size_t)g.k * g.r * g.s * g.c, P.splits / P.cl, g.alpha, stream);
     return cudaGetLastError();
 }
 

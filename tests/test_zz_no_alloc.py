@@ -50,7 +50,7 @@ def test_static_scratch_entry_matches_workspace_entry_twice(dtype, layer):
 
 
 def test_static_scratch_entry_rejects_problems_beyond_its_limit():
-    big = ConvLayer("too big", 128, 64, 32, 32, 64, 3, 3, 1, 1)       # over a hundred split partials of 147 KB
+    big = ConvLayer("too big", 4096, 64, 2, 2, 512, 3, 3, 1, 1)       # its transposed copy of dY alone is 16 MiB
     d = B.make_desc(big, torch.bfloat16)
     assert B.gaconv_workspace_size(d, B.METHOD_EXACT) > B.gaconv_static_scratch_bytes()
     with pytest.raises(B.GaconvError) as e:
