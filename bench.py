@@ -236,8 +236,8 @@ def main():
     from paper_1908_05460_b200 import inputs as I
     from paper_1908_05460_b200 import build as build_mod
 
-    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_1908_05460_b200 import dist_util
+    rank, world, local = dist_util.env_rank()
     if rank == 0:
         build_mod.build()
     torch.cuda.set_device(local)
@@ -322,12 +322,9 @@ def main():
     if rank == 0:
         time.sleep(0.2)
     clocks = sampler.stop() if rank == 0 else None
-    tt = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    ms_step = float(tt.item()) / args.steps
+    ms_step = dist_util.max_over_ranks(ms_total, "cuda") / args.steps      # slowest rank decides
     passes = len(slots)
-    value = ms_step * 1e3 / (passes * world)
+    value = dist_util.us_per_layer(ms_step, passes, world)
 
     # ---- per-layer timing on the launching stream ----
     # streamed: a CUDA graph of back-to-back launches of one layer, each on its own copy of the inputs,
@@ -414,7 +411,10 @@ def main():
                 "kernel": "top-1 select+gather", "launches": len(table)}
     roof["frac"] = roof["achieved"] / roof["peak"] if table else None
     roof["peak_source"] = peaks["source"]
-    roof["traffic"] = None
+    # DRAM bytes of one launch from the committed ncu capture of this kernel family (profiles/): the exact
+    # fp32 kernel on 16->16@32x32, N=128 moved 16.85 MB for 16.79 MB of algorithmic bytes (no re-reads)
+    roof["traffic"] = {"bytes_per_launch": 16845056, "algorithmic_bytes": 16786432, "layer": "16->16@32 f32 N=128",
+                       "source": "profiles/direct_tiled_f32_16x16_32x32_n128.md"} if roof.get("kernel") == "exact dW" else None
 
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
     e2e = None
@@ -432,10 +432,8 @@ def main():
             e2e_step(t)
         ev1.record()
         barrier()
-        ms_e = torch.tensor([ev0.elapsed_time(ev1) / k2], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(ms_e, op=dist.ReduceOp.MAX)
-        e2e = {"value": float(ms_e.item()) * 1e3 / (passes * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        ms_e = dist_util.max_over_ranks(ev0.elapsed_time(ev1) / k2, "cuda")
+        e2e = {"value": dist_util.us_per_layer(ms_e, passes, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": k2}
 
     if rank != 0:
