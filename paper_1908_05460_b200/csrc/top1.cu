@@ -425,8 +425,8 @@ cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Ge
     int cl = 1;
     while (cl * 2 <= 8 && cl * 2 <= g.n) cl *= 2;
     // fewer, fatter CTAs when there are already plenty of channels: the whole grid should be resident
-    // at once (clusters are placed GPC by GPC), i.e. about two CTAs per SM
-    while (cl > 1 && (long long)cl * g.k > 148 * 2) cl /= 2;
+    // at once (four CTAs of 64 registers x 256 threads fit an SM)
+    while (cl > 1 && (long long)cl * g.k > 148 * 4) cl /= 2;
     const int ipc = (g.n + cl - 1) / cl;
     const MapScanShape m = map_scan_shape(g);
     if (g.bf16) {
