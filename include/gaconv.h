@@ -49,8 +49,10 @@ typedef enum { GACONV_METHOD_EXACT = -1, GACONV_METHOD_ZERO = 0, GACONV_METHOD_R
                GACONV_METHOD_TOP1 = 2 } gaconv_method_t;
 /* arithmetic of the exact contraction */
 typedef enum {
-    GACONV_MATH_DEFAULT = 0,   /* bf16 inputs: bf16 tensor cores, fp32 accumulate; fp32 inputs: fp32-accurate */
-    GACONV_MATH_TF32 = 1       /* fp32 inputs only: one TF32 tensor-core pass (operands cut to 10 mantissa bits) */
+    GACONV_MATH_DEFAULT = 0,   /* bf16 inputs: bf16 tensor cores, fp32 accumulate; fp32 inputs: fp32-accurate
+                                  (three TF32 tensor-core passes on split operands, or the FP32 pipes)          */
+    GACONV_MATH_TF32 = 1       /* fp32 inputs only: one TF32 tensor-core pass (operands cut to 10 mantissa bits);
+                                  GACONV_ERR_UNSUPPORTED for shapes without a tensor-core kernel                 */
 } gaconv_math_t;
 /* kernel family; AUTO picks the fastest that supports the shape */
 typedef enum { GACONV_ALGO_AUTO = 0, GACONV_ALGO_DIRECT = 1, GACONV_ALGO_TENSOR = 2 } gaconv_algo_t;

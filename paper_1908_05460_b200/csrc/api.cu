@@ -168,8 +168,9 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
-    if (desc->math == GACONV_MATH_TF32) return GACONV_ERR_UNSUPPORTED;
     const ExactLayout L = exact_layout(g);
+    const bool mma_ok = direct_mma_supported(g, L.dp);
+    if (desc->math == GACONV_MATH_TF32 && !mma_ok) return GACONV_ERR_UNSUPPORTED;
     if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
     st = check_ws(desc, L.total);
     if (st != GACONV_OK) return st;
@@ -178,6 +179,11 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
         cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
                                   reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
                                   static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    }
+    if (mma_ok && (desc->algo != GACONV_ALGO_DIRECT || desc->math == GACONV_MATH_TF32)) {
+        cudaError_t e = launch_direct_mma(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), reinterpret_cast<uint32_t*>(ws),
+                                          g, L.dp, desc->math != GACONV_MATH_TF32, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     cudaError_t e = launch_direct(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off),

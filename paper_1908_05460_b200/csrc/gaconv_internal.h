@@ -71,6 +71,11 @@ DirectPlan plan_direct(const Geom& g);
 cudaError_t launch_direct(const void* x, const void* dy, float* dw, float* partial, uint32_t* status,
                           const Geom& g, const DirectPlan& plan, cudaStream_t stream);
 
+// ---- exact filter gradient, fp32 inputs on mma.sync with split TF32 operands (3 passes: fp32 accuracy) ----
+bool direct_mma_supported(const Geom& g, const DirectPlan& plan);
+cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* partial, uint32_t* status, const Geom& g,
+                              const DirectPlan& plan, bool three_pass, cudaStream_t stream);
+
 // ---- exact filter gradient on tcgen05 tensor cores (bf16, NHWC X, shapes its tiling covers) ----
 struct TcPlan {
     size_t partial_bytes;

@@ -281,3 +281,41 @@ def test_tensor_core_exact_matches_oracle_and_direct(li):
     scale = np.maximum(np.abs(direct), 1e-3 * np.abs(direct).max())
     assert np.max(np.abs(got - direct) / scale) < 1e-2
     np.testing.assert_array_equal(got, g.exact())                      # reproducible bit for bit
+
+
+# ---- fp32 inputs: warp-level tensor-core path with split TF32 operands, and the FP32-pipe kernel ----
+MMA_SHAPES = [
+    ConvLayer("mma 16->16@32", 6, 16, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("mma 32->32@16 two c tiles", 5, 32, 16, 16, 32, 3, 3, 1, 1),
+    ConvLayer("mma 64->64@8", 9, 64, 8, 8, 64, 3, 3, 1, 1),
+    ConvLayer("mma stride 2", 4, 16, 32, 32, 32, 3, 3, 2, 1),
+    ConvLayer("mma ragged channels", 3, 24, 16, 16, 20, 3, 3, 1, 1),
+    ConvLayer("mma 1x1", 4, 32, 16, 16, 48, 1, 1, 1, 0),
+    ConvLayer("mma c8", 7, 8, 32, 32, 16, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("li", range(len(MMA_SHAPES)), ids=[l.name for l in MMA_SHAPES])
+def test_fp32_exact_split_tf32_and_fp32_pipes(li):
+    layer = MMA_SHAPES[li]
+    x, dy = _inputs(layer, torch.float32, 300 + li)
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.5)
+    auto = GpuLayer(layer, torch.float32, x, dy, alpha=0.5)                       # split-TF32 tensor path
+    got = auto.exact()
+    assert norm_err(got, ref, dn) <= TOL_F32
+    np.testing.assert_array_equal(got, auto.exact())
+    pipes = GpuLayer(layer, torch.float32, x, dy, alpha=0.5, algo=B.ALGO_DIRECT)   # FP32 pipes
+    assert norm_err(pipes.exact(), ref, dn) <= TOL_F32
+    one = GpuLayer(layer, torch.float32, x, dy, alpha=0.5, math=B.MATH_TF32)      # one TF32 pass: its own, looser class
+    e1 = norm_err(one.exact(), ref, dn)
+    assert e1 <= 4e-3
+    assert B.gaconv_poll_async_status(auto.desc) == B.OK
+
+
+def test_tf32_mode_is_refused_where_it_has_no_kernel():
+    layer = ConvLayer("5x5", 2, 16, 16, 16, 16, 5, 5, 1, 2)
+    x, dy = _inputs(layer, torch.float32, 320)
+    g = GpuLayer(layer, torch.float32, x, dy, math=B.MATH_TF32)
+    with pytest.raises(B.GaconvError) as e:
+        g.exact()
+    assert e.value.status == B.ERR_UNSUPPORTED
