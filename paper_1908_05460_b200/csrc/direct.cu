@@ -144,6 +144,7 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
         tma_load_3d(dst, &map_dy, full, p0 * g.q, k0, n);
         tma_load_4d(dst + TK * npx * 4, &map_x, full, c0, -g.pad_w, p0 * g.stride_h - g.pad_h, n);
     };
+    if (STAGING != 1) pdl_wait_prior_grid();
     if (STAGING == 1) {
         if (threadIdx.x == 0) {
             s_fail = 0;
@@ -151,6 +152,7 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncthreads();
+        pdl_wait_prior_grid();
         if (threadIdx.x == 0 && it_begin < it_end) tma_issue(it_begin, 0);
     } else if (it_begin < it_end) {
         stage_item<T, false, TK, TC>(x, dy, smem, smem + TK * dys, g, pl, it_begin, k0, c0, dys, win_h, win_w);
@@ -244,6 +246,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 direct_element_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g)
 {
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
     const long long total = (long long)g.k * g.r * g.s * g.c;
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= total) return;
@@ -320,11 +324,12 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_
             use_tma = false;
     }
     bool done = false;
+    cudaError_t launch_err = cudaSuccess;
 #define GACONV_DIRECT_LAUNCH(ST, RR, A, B, C, D)                                                                                 \
     {                                                                                                                            \
         auto kern = direct_tiled_kernel<T, ST, RR, RR, A, B, C, D>;                                                              \
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                \
-        kern<<<grid, kThreads, smem, stream>>>(x, dy, dw, partial, status, map_dy, map_x, g, pl);                                \
+        launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), x, dy, dw, partial, status, map_dy, map_x, g, pl); \
     }
 #define GACONV_DIRECT_CASE(RR, A, B, C, D)                                                                     \
     if (!done && g.r == RR && v.tkt == A && v.tct == B && v.otk == C && v.otc == D) {                          \
@@ -342,8 +347,7 @@ cudaError_t launch_t(const T* x, const T* dy, float* dw, float* partial, uint32_
 #undef GACONV_DIRECT_LAUNCH
     if (!done) return cudaErrorInvalidValue;
     note_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (launch_err != cudaSuccess) return launch_err;
     if (pl.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.c * g.r * g.s, pl.splits, g.alpha, stream);
     return cudaSuccess;
 }

@@ -76,6 +76,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait_prior_grid();
     if (threadIdx.x == 0 && it_begin < it_end) tma_issue(it_begin, 0);
 
     int stage = 0;
@@ -191,11 +192,12 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     size_t smem = 2 * stage > red ? 2 * stage : red;
     smem += 1024;
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
+    cudaError_t launch_err = cudaErrorInvalidValue;
 #define GACONV_MMA_CASE(RR, TP)                                                                                          \
     if (g.r == RR && three_pass == TP) {                                                                                 \
         auto kern = direct_mma_kernel<RR, RR, TP>;                                                                       \
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
-        kern<<<grid, kThreads, smem, stream>>>(dw, partial, status, map_dy, map_x, g, pl);                               \
+        launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), dw, partial, status, map_dy, map_x, g, pl); \
     }
     GACONV_MMA_CASE(1, true)
     GACONV_MMA_CASE(1, false)
@@ -203,8 +205,7 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     GACONV_MMA_CASE(3, false)
 #undef GACONV_MMA_CASE
     note_launch();
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (launch_err != cudaSuccess) return launch_err;
     if (pl.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.c * g.r * g.s, pl.splits, g.alpha, stream);
     return cudaSuccess;
 }

@@ -13,6 +13,8 @@ namespace {
 
 __global__ void __launch_bounds__(256) zero_kernel(float* __restrict__ dw, size_t count)
 {
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t nvec = count / 4;
     float4* v = reinterpret_cast<float4*>(dw);
@@ -50,6 +52,7 @@ __device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float& z0, 
 __global__ void __launch_bounds__(256)
 random_kernel(float* __restrict__ dw, size_t count, Geom g, uint32_t key0, uint32_t key1, float std, bool contiguous)
 {
+    pdl_release_next_grid();
     const size_t j = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (4 * j >= count) return;
     uint32_t c[4] = {(uint32_t)j, 0u, 0u, 0u};
@@ -62,6 +65,7 @@ random_kernel(float* __restrict__ dw, size_t count, Geom g, uint32_t key0, uint3
     float z[4];
     box_muller(c[0], c[1], z[0], z[1]);
     box_muller(c[2], c[3], z[2], z[3]);
+    pdl_wait_prior_grid();      // the values need no memory; only the stores wait for the previous kernel
     if (contiguous && 4 * j + 3 < count) {
         reinterpret_cast<float4*>(dw)[j] = make_float4(std * z[0], std * z[1], std * z[2], std * z[3]);
         return;
@@ -93,9 +97,8 @@ cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream)
     size_t blocks = (count / 4 + 255) / 256;
     if (blocks < 1) blocks = 1;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    zero_kernel<<<(unsigned)blocks, 256, 0, stream>>>(dw, count);
     note_launch();
-    return cudaGetLastError();
+    return launch_kernel(zero_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, dim3(1, 1, 1), dw, count);
 }
 
 cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cudaStream_t stream)
@@ -103,10 +106,9 @@ cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cu
     const size_t count = (size_t)g.k * g.c * g.r * g.s;
     const size_t threads = (count + 3) / 4;
     const bool contiguous = (g.ws_s == 1 && g.ws_r == g.s && g.ws_c == (long long)g.r * g.s);
-    random_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(dw, count, g, (uint32_t)seed,
-                                                                          (uint32_t)(seed >> 32), std, contiguous);
     note_launch();
-    return cudaGetLastError();
+    return launch_kernel(random_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, stream, dim3(1, 1, 1), dw, count, g,
+                         (uint32_t)seed, (uint32_t)(seed >> 32), std, contiguous);
 }
 
 }  // namespace gaconv

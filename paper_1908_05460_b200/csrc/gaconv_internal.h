@@ -7,6 +7,8 @@
 
 #include "gaconv.h"
 
+#include <utility>
+
 namespace gaconv {
 
 // ---- workspace layout -------------------------------------------------------------------------
@@ -18,6 +20,37 @@ constexpr int    kWsNumCounters   = 4096;
 constexpr size_t kWsDataOffset    = kWsCounterOffset + sizeof(uint32_t) * kWsNumCounters;
 
 void note_launch(int count = 1);   // bookkeeping behind gaconv_launch_count()
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization allowed and starts
+// with pdl_release_next_grid(): the next kernel in the stream may then be scheduled while this one is
+// still running, and do its own set-up (barrier init, tensor-memory allocation) early.  Before its
+// first access to global memory every kernel executes pdl_wait_prior_grid(), which returns only when
+// the previous kernel has completed and its writes are visible -- so results never depend on it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_release_next_grid() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 dim3 cluster, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster.x * cluster.y * cluster.z > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster.x; attr[n].val.clusterDim.y = cluster.y; attr[n].val.clusterDim.z = cluster.z;
+        ++n;
+    }
+    cfg.attrs = attr; cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

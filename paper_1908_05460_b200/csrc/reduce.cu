@@ -23,6 +23,9 @@ __global__ void __launch_bounds__(32 * kReduceWarps)
 reduce_splits_kernel(const V* __restrict__ partial, V* __restrict__ dw, size_t count, int splits, float alpha)
 {
     __shared__ V sm[kReduceWarps][32];
+    // no early release here: the kernels that follow are sized as one wave, and placing their CTAs while
+    // this kernel's large blocks still hold some SMs unbalances that wave
+    pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + lane;
     V acc = vzero<V>();
@@ -48,15 +51,14 @@ cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int spl
     // as many warps per block as there are splits to share out (a power of two, at most 32)
     int warps = 1;
     while (warps < splits && warps < kReduceWarps) warps *= 2;
+    note_launch();
     if (count % 4 == 0) {
         const size_t c4 = count / 4;
-        reduce_splits_kernel<float4><<<(unsigned)((c4 + 31) / 32), 32 * warps, 0, stream>>>(
-            reinterpret_cast<const float4*>(partial), reinterpret_cast<float4*>(dw), c4, splits, alpha);
-    } else {
-        reduce_splits_kernel<float><<<(unsigned)((count + 31) / 32), 32 * warps, 0, stream>>>(partial, dw, count, splits, alpha);
+        return launch_kernel(reduce_splits_kernel<float4>, dim3((unsigned)((c4 + 31) / 32)), dim3(32 * warps), 0, stream, dim3(1, 1, 1),
+                             reinterpret_cast<const float4*>(partial), reinterpret_cast<float4*>(dw), c4, splits, alpha);
     }
-    note_launch();
-    return cudaGetLastError();
+    return launch_kernel(reduce_splits_kernel<float>, dim3((unsigned)((count + 31) / 32)), dim3(32 * warps), 0, stream, dim3(1, 1, 1),
+                         partial, dw, count, splits, alpha);
 }
 
 }  // namespace gaconv

@@ -126,6 +126,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // reduction block, aliases the stages
     const int red_stride = P.rc * nmma + 4;
 
+    pdl_release_next_grid();
     if (threadIdx.x == 0) {
         for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), P.issuers); }
         mbar_init(smem_u32(&bar_acc), P.issuers);
@@ -140,6 +141,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = s_tmem_base;
+    pdl_wait_prior_grid();     // set-up done; from here on global memory of the previous kernel is read and written
     long long* tl = (P.timeline && blockIdx.x == 0 && blockIdx.y == 0) ? reinterpret_cast<long long*>(status + 16) : nullptr;
     if (tl && threadIdx.x == 0) tl[0] = clock64();
 
@@ -355,6 +357,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
 __global__ void __launch_bounds__(256)
 transpose_dy_kernel(const __nv_bfloat16* __restrict__ dy, __nv_bfloat16* __restrict__ dyt, int n, int k, int pq)
 {
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
     const size_t total = (size_t)n * k * pq;
     const size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // output index: ((n*pq + j)*k + kk)
     if (o >= total) return;
@@ -510,8 +514,9 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     CUtensorMap map_dy, map_x;
     if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) with 64-channel boxes
         const size_t total = (size_t)g.n * g.k * pq;
-        transpose_dy_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.n, g.k, pq);
+        if (launch_kernel(transpose_dy_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, stream, dim3(1, 1, 1),
+                          static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.n, g.k, pq) != cudaSuccess)
+            return cudaErrorLaunchFailure;
         note_launch();
         cuuint64_t dims[3] = {(cuuint64_t)g.k, (cuuint64_t)pq, (cuuint64_t)g.n};
         cuuint64_t strides[2] = {(cuuint64_t)g.k * 2, (cuuint64_t)g.k * pq * 2};
@@ -558,13 +563,8 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
             if (err == cudaSuccess) configured = smem;                                                             \
         }                                                                                                          \
         if (err == cudaSuccess) {                                                                                  \
-            cudaLaunchConfig_t cfg = {};                                                                           \
-            cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = stream;        \
-            cudaLaunchAttribute attr[1];                                                                           \
-            attr[0].id = cudaLaunchAttributeClusterDimension;                                                      \
-            attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = P.cl; attr[0].val.clusterDim.z = 1;           \
-            cfg.attrs = attr; cfg.numAttrs = 1;                                                                    \
-            err = cudaLaunchKernelEx(&cfg, exact_tc_kernel<RR, KK>, map_dy, map_x, dw, partial, counters, status, P); \
+            err = launch_kernel(exact_tc_kernel<RR, KK>, grid, dim3(256), smem, stream, dim3(1, P.cl, 1), map_dy, map_x, dw, \
+                                partial, counters, status, P);                                                    \
         }                                                                                                          \
     }
     GACONV_TC_CASE(3, 4)

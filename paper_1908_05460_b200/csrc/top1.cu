@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(256)
 select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __restrict__ sum,
               T* __restrict__ dy_sparse, long long num_maps, int pq, int G)
 {
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
     const int lane = threadIdx.x & 31;
     const int sub = lane & (G - 1);
     const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -160,6 +162,7 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    pdl_wait_prior_grid();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int rsc = g.r * g.s * g.c;
     float* s_part = reinterpret_cast<float*>(smem_raw);                 // [rsc]
@@ -267,6 +270,8 @@ gather_kernel(const T* __restrict__ x, const int32_t* __restrict__ idx, const fl
               float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters, Geom g,
               int chunks, int ipc)
 {
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
     extern __shared__ int smem_i[];
     int* s_h0 = smem_i;                       // top-left input row of each image's patch
     int* s_w0 = smem_i + ipc;
@@ -406,16 +411,7 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cl, g.k);
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, top1_fused_kernel<T, VEC>, x, dy, dw, g, ipc, G, vec_x);
+    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(256), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x);
     note_launch();
     return e;
 }
