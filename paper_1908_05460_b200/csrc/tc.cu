@@ -47,8 +47,9 @@ __device__ __forceinline__ void umma_bf16_acc(uint32_t d_tmem, uint64_t adesc, u
 __device__ __forceinline__ float4 ld_dsmem_f4(uint32_t local_addr, uint32_t rank) {
     uint32_t remote;
     float4 v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    // not volatile: the blocks are stable between the two cluster barriers, so the compiler may batch these loads
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote));
     return v;
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -315,6 +316,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int cl = P.cl, rank = cl > 1 ? (int)cluster.block_rank() : 0;
     const int groups_per_tile = P.splits / cl, cgroup = split / cl;
     if (cl > 1) cluster.sync();
+    if (tl && threadIdx.x == 0) tl[5] = clock64();
     const int rows = min(P.m, g.k - k0), cols = P.rc * nmma;
     const int q_per_row = cols >> 2, quads = rows * q_per_row;
     const int slice = (quads + cl - 1) / cl;
@@ -335,11 +337,14 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         for (int f = f_begin + (int)threadIdx.x; f < f_end; f += blockDim.x) {
             const int row = f / q_per_row, col = (f - row * q_per_row) << 2;
             const float* src = red + row * red_stride + col;
-            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int rk = 0; rk < cl; ++rk) {
-                const float4 v = cl > 1 ? ld_dsmem_f4(smem_u32(src), (uint32_t)rk) : *reinterpret_cast<const float4*>(src);
-                t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
-            }
+            float4 v[4];                                            // all ranks' pieces first (cl <= 4), then the sum in rank order
+#pragma unroll
+            for (int rk = 0; rk < 4; ++rk)
+                v[rk] = rk >= cl ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                 : cl > 1 ? ld_dsmem_f4(smem_u32(src), (uint32_t)rk) : *reinterpret_cast<const float4*>(src);
+            float4 t = v[0];
+#pragma unroll
+            for (int rk = 1; rk < 4; ++rk) { t.x += v[rk].x; t.y += v[rk].y; t.z += v[rk].z; t.w += v[rk].w; }
             int c, valid;
             const size_t off = out_offset(f, c, valid);
             if (vec && valid == 4) {
@@ -350,7 +355,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             }
         }
     }
+    if (tl && threadIdx.x == 0) tl[6] = clock64();
     if (cl > 1) cluster.sync();      // peers may still be reading this CTA's block
+    if (tl && threadIdx.x == 0) tl[7] = clock64();
 }
 
 // dYt[n][j][k] = dY[n][k][j] for maps of fewer than 16 pixels (the map is too short for a TMA row).
@@ -402,9 +409,12 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.m = (g.k <= 64 || g.c >= 64) ? 64 : 128;
     // Many output channels and wide inputs: one filter row per CTA, so that a full-rate M = 128 MMA with a
     // 64-channel (128-byte row) B tile fits tensor memory (S*64 columns) and the epilogue block shrinks.
-    P.rsplit = (g.k >= 128 && g.c >= 64 && g.r > 1 && env_int("GACONV_TC_RSPLIT", 1)) ? 1 : 0;
+    // The same split also pays for K <= 64 with 64-channel tiles: the block a CTA has to reduce across its
+    // cluster shrinks from 64 x R*S*64 floats (147 KB for 3x3) to a third, and that reduction, not the MMAs,
+    // is what a small layer spends its time on.
+    P.rsplit = (g.c >= 64 && g.r > 1 && env_int("GACONV_TC_RSPLIT", 1)) ? 1 : 0;
     P.rc = P.rsplit ? 1 : g.r;
-    if (P.rsplit) P.m = 128;
+    if (P.rsplit) P.m = g.k <= 64 ? 64 : 128;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     P.tiny = tiny ? 1 : 0;
     P.by_image = small_map ? 1 : 0;
@@ -473,6 +483,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
     int cl = 1;
     while (cl * 2 <= 8 && tiles * cl * 2 <= 128 && cl * 2 <= P.chunks) cl *= 2;
+    if (cl > 4) cl = 4;      // the reduction loop holds one piece per rank in registers
     if (env_int("GACONV_TC_CLUSTER", 4) < cl) cl = env_int("GACONV_TC_CLUSTER", 4) < 1 ? 1 : env_int("GACONV_TC_CLUSTER", 4);
     int splits = env_int("GACONV_TC_SPLITS", 0);
     if (splits <= 0) {
