@@ -157,7 +157,7 @@ template <> __device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __
 //            distributed shared memory, in rank order, and writes alpha * total to dW.
 // No global scratch, no atomics; the order of every sum is fixed.
 template <typename T, bool VEC>
-__global__ void __launch_bounds__(256, 4)
+__global__ void __launch_bounds__(512, 2)
 top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x)
 {
     namespace cg = cooperative_groups;
@@ -403,7 +403,10 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     const int rsc = g.r * g.s * g.c;
     const bool vec_x = g.xs_c == 1 && g.c % 4 == 0;
     int nj = 1;
-    while (nj * 2 * (rsc / (vec_x ? 4 : 1)) <= 256 && nj * 2 <= 16) nj *= 2;
+    // 512 threads (two CTAs per SM) where the grid still fits in one wave and the scan would otherwise need
+    // two passes over the CTA's maps; measured: helps 32-channel layers, neutral or worse for 16 and 64
+    const int threads = (g.k >= 32 && (long long)cl * g.k <= 148 * 2) ? 512 : 256;
+    while (nj * 2 * (rsc / (vec_x ? 4 : 1)) <= threads && nj * 2 <= 16) nj *= 2;
     const size_t smem = (size_t)rsc * sizeof(float) * (nj > 1 ? 1 + nj : 1) + (size_t)ipc * 12 + 16;
     static size_t configured = 0;
     if (smem > 48 * 1024 && smem > configured) {
@@ -411,7 +414,7 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(256), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x);
+    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x);
     note_launch();
     return e;
 }
