@@ -78,7 +78,7 @@ Top1Layout top1_layout(const Geom& g)
     return L;
 }
 
-struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; bool tc_ok; };
+struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; StemPlan sp; bool tc_ok, stem_ok; };
 ExactLayout exact_layout(const Geom& g)
 {
     ExactLayout L;
@@ -87,6 +87,8 @@ ExactLayout exact_layout(const Geom& g)
     L.partial_off = kWsDataOffset;
     size_t partial = L.dp.partial_bytes;
     if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
+    L.stem_ok = plan_stem(g, &L.sp);
+    if (L.stem_ok && L.sp.partial_bytes > partial) partial = L.sp.partial_bytes;
     L.scratch_off = align_up(L.partial_off + partial, 256);
     L.total = align_up(L.scratch_off + (L.tc_ok ? L.tp.scratch_bytes : 0), 256);
     return L;
@@ -179,6 +181,11 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
         cudaError_t e = launch_tc(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
                                   reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
                                   static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    }
+    if (L.stem_ok && desc->algo != GACONV_ALGO_DIRECT && desc->math == GACONV_MATH_DEFAULT) {
+        cudaError_t e = launch_stem(x, dy, dw, reinterpret_cast<float*>(ws + L.partial_off), reinterpret_cast<uint32_t*>(ws), L.sp,
+                                    static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     }
     if (mma_ok && (desc->algo != GACONV_ALGO_DIRECT || desc->math == GACONV_MATH_TF32)) {

@@ -364,8 +364,11 @@ DirectPlan plan_direct(const Geom& g)
     pl.tiles_c = (g.c + tc - 1) / tc;
     pl.bq = g.q < 32 ? g.q : 32;
     pl.bp = 1;
-    while (pl.bp * 2 <= g.p && pl.bp * 2 * pl.bq <= 128 && smem_for(g, v, pl.bp * 2, pl.bq) <= 64 * 1024) pl.bp *= 2;
-    while (pl.bq > 1 && smem_for(g, v, pl.bp, pl.bq) > 64 * 1024) pl.bq /= 2;
+    // few input channels: the items are cheap and staged by the threads themselves, so a CTA takes its whole
+    // share as one or two large items (one exposed load latency instead of four)
+    const int max_px = g.c <= 4 ? 512 : 128;
+    while (pl.bp * 2 <= g.p && pl.bp * 2 * pl.bq <= max_px && smem_for(g, v, pl.bp * 2, pl.bq) <= 96 * 1024) pl.bp *= 2;
+    while (pl.bq > 1 && smem_for(g, v, pl.bp, pl.bq) > 96 * 1024) pl.bq /= 2;
     pl.bands_p = (g.p + pl.bp - 1) / pl.bp;
     pl.bands_q = (g.q + pl.bq - 1) / pl.bq;
     // vector fast paths: bands of whole rows whose pixel runs start on a 4-element boundary; NHWC with

@@ -109,6 +109,15 @@ bool direct_mma_supported(const Geom& g, const DirectPlan& plan);
 cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* partial, uint32_t* status, const Geom& g,
                               const DirectPlan& plan, bool three_pass, cudaStream_t stream);
 
+// ---- exact filter gradient for layers with at most four input channels (stems), mma.sync over flattened image rows ----
+struct StemPlan {
+    size_t partial_bytes;
+    alignas(8) unsigned char opaque[256];   // kernel parameters, private to stem_mma.cu
+};
+bool plan_stem(const Geom& g, StemPlan* plan);
+cudaError_t launch_stem(const void* x, const void* dy, float* dw, float* partial, uint32_t* status, const StemPlan& plan,
+                        cudaStream_t stream);
+
 // ---- exact filter gradient on tcgen05 tensor cores (bf16, NHWC X, shapes its tiling covers) ----
 struct TcPlan {
     size_t partial_bytes;

@@ -319,3 +319,31 @@ def test_tf32_mode_is_refused_where_it_has_no_kernel():
     with pytest.raises(B.GaconvError) as e:
         g.exact()
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+# ---- few-channel (stem) layers: mma.sync over flattened image rows, both dtypes, against oracle and FP32 pipes ----
+STEM_SHAPES = [
+    ConvLayer("stem 3->16@32", 6, 3, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("stem 3->64@32", 3, 3, 32, 32, 64, 3, 3, 1, 1),
+    ConvLayer("stem 5x5 3->64@32", 3, 3, 32, 32, 64, 5, 5, 1, 2, x_dist="uniform_pm1"),
+    ConvLayer("stem 4 channels k20", 5, 4, 16, 16, 20, 3, 3, 1, 1),
+    ConvLayer("stem stride 2", 4, 3, 32, 32, 24, 3, 3, 2, 1),
+    ConvLayer("stem 1 channel", 7, 1, 32, 32, 8, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("li", range(len(STEM_SHAPES)), ids=[l.name for l in STEM_SHAPES])
+def test_stem_layers(li, dtype):
+    layer = STEM_SHAPES[li]
+    x, dy = _inputs(layer, dtype, 400 + li)
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 2.0)
+    auto = GpuLayer(layer, dtype, x, dy, alpha=2.0)
+    got = auto.exact()
+    assert norm_err(got, ref, dn) <= (TOL_F32 if dtype == torch.float32 else 1e-4)
+    np.testing.assert_array_equal(got, auto.exact())
+    pipes = GpuLayer(layer, dtype, x, dy, alpha=2.0, algo=B.ALGO_DIRECT)
+    assert norm_err(pipes.exact(), ref, dn) <= tol(dtype)
+    kcrs = GpuLayer(layer, dtype, x, dy, alpha=2.0, dw_layout=B.DW_KCRS)
+    assert norm_err(kcrs.exact(), ref, dn) <= tol(dtype)
+    assert B.gaconv_poll_async_status(auto.desc) == B.OK
