@@ -10,9 +10,9 @@
 // range of work items (an item = one image's band of whole output rows); the dY band and the X window
 // arrive as fp32 TMA boxes in two shared-memory stages.  Per 8 pixels (one MMA k-step) a warp loads the
 // 16x8 dY fragment once and, for each tap and each half of the 16 channels, an 8x8 X fragment, splits
-// both in registers and issues three MMAs into the tap's accumulator.  The four warps of a CTA take
-// the k-steps round-robin; their accumulators are added through shared memory in warp order, and the
-// splits by reduce_splits().
+// both in registers and issues three MMAs into the tap's accumulator.  For 1x1 and 3x3 filters the four
+// warps of a CTA take the k-steps round-robin and their accumulators are added through shared memory in
+// warp order; for 5x5 they split the 25 taps instead (register budget).  Splits: reduce_splits().
 //   dY box: 32 pixels x 16 channels with the 128-byte TMA swizzle, so that the eight k-rows a fragment
 //   load touches fall in different banks.
 #include "gaconv_internal.h"
@@ -40,7 +40,13 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
                   const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
                   Geom g, DirectPlan pl)
 {
-    constexpr int TAPS = R * S, NT = TAPS * 2;          // n-tiles of 8 channels: tap-major, channel half minor
+    constexpr int TAPS = R * S;
+    // Up to 9 taps: every warp holds all taps and the warps split the k-steps (their accumulators are added at
+    // the end).  More taps (5x5): the accumulators would not fit the register file, so the warps split the
+    // TAPS instead -- each runs all k-steps for its own taps, and no cross-warp sum is needed.
+    constexpr bool SPLIT_TAPS = TAPS > 9;
+    constexpr int TPW = SPLIT_TAPS ? (TAPS + kWarps - 1) / kWarps : TAPS;   // taps per warp
+    constexpr int NT = TPW * 2;                          // n-tiles of 8 channels: tap-major, channel half minor
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[2];
     __shared__ volatile int s_fail;
@@ -59,6 +65,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
     float acc[NT][4];
 #pragma unroll
     for (int i = 0; i < NT; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+    const int tap_lo = SPLIT_TAPS ? warp * TPW : 0;      // first tap of this warp
 
     const int per = (pl.items + pl.splits - 1) / pl.splits;
     const int it_begin = split * per, it_end = min(pl.items, (split + 1) * per);
@@ -91,7 +98,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
         const uint8_t* s_dy = smem + stage * stage_bytes;
         const float* s_x = reinterpret_cast<const float*>(s_dy + dy_bytes);
 
-        for (int ks = warp; ks < npx / 8; ks += kWarps) {
+        for (int ks = SPLIT_TAPS ? 0 : warp; ks < npx / 8; ks += SPLIT_TAPS ? 1 : kWarps) {
             const int px0 = ks * 8;
             // ---- A fragment: dY[k = gq (+8)][px0 + tq (+4)], from the swizzled box ----
             uint32_t a_big[4], a_small[4];
@@ -111,23 +118,24 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
             const float* xrow = s_x + ((pp * g.stride_h) * win_w + (qq + tq) * g.stride_w) * TC + gq;
             const int px4 = 4 * g.stride_w * TC;                 // four pixels further along the row
 #pragma unroll
-            for (int r = 0; r < R; ++r)
+            for (int i = 0; i < TPW; ++i) {
+                const int tap = tap_lo + i;
+                if (SPLIT_TAPS && tap >= TAPS) break;
+                const int r = SPLIT_TAPS ? tap / S : i / S, s = SPLIT_TAPS ? tap % S : i % S;
+                const float* xt = xrow + (r * win_w + s) * TC;
 #pragma unroll
-                for (int s = 0; s < S; ++s) {
-                    const float* xt = xrow + (r * win_w + s) * TC;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const float v0 = xt[h * 8], v1 = xt[h * 8 + px4];
-                        const uint32_t b0 = to_tf32(v0), b1 = to_tf32(v1);
-                        float (&d)[4] = acc[(r * S + s) * 2 + h];
-                        if (THREE_PASS) {
-                            const uint32_t s0 = to_tf32(v0 - __uint_as_float(b0)), s1 = to_tf32(v1 - __uint_as_float(b1));
-                            mma_tf32(d, a_small, b0, b1);
-                            mma_tf32(d, a_big, s0, s1);
-                        }
-                        mma_tf32(d, a_big, b0, b1);
+                for (int h = 0; h < 2; ++h) {
+                    const float v0 = xt[h * 8], v1 = xt[h * 8 + px4];
+                    const uint32_t b0 = to_tf32(v0), b1 = to_tf32(v1);
+                    float (&d)[4] = acc[i * 2 + h];
+                    if (THREE_PASS) {
+                        const uint32_t s0 = to_tf32(v0 - __uint_as_float(b0)), s1 = to_tf32(v1 - __uint_as_float(b1));
+                        mma_tf32(d, a_small, b0, b1);
+                        mma_tf32(d, a_big, s0, s1);
                     }
+                    mma_tf32(d, a_big, b0, b1);
                 }
+            }
         }
         __syncthreads();    // everyone is done with this stage before it is refilled
     }
@@ -136,13 +144,14 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
     // s_red[warp][k][tap][c]: thread (gq, tq) holds rows gq, gq+8 and columns 2*tq, 2*tq+1 of each n-tile
     float* s_red = reinterpret_cast<float*>(smem);
     constexpr int BLK = TK * TAPS * TC;
+    constexpr int SLOTS = SPLIT_TAPS ? 1 : kWarps;       // split taps: the warps own disjoint columns of one block
 #pragma unroll
     for (int i = 0; i < NT; ++i) {
-        const int tap = i >> 1, cbase = (i & 1) * 8 + 2 * tq;
-        float* w0 = s_red + warp * BLK + (gq * TAPS + tap) * TC + cbase;
-        float* w1 = s_red + warp * BLK + ((gq + 8) * TAPS + tap) * TC + cbase;
-        *reinterpret_cast<float2*>(w0) = make_float2(acc[i][0], acc[i][1]);
-        *reinterpret_cast<float2*>(w1) = make_float2(acc[i][2], acc[i][3]);
+        const int tap = tap_lo + (i >> 1), cbase = (i & 1) * 8 + 2 * tq;
+        if (SPLIT_TAPS && tap >= TAPS) continue;
+        float* base = s_red + (SPLIT_TAPS ? 0 : warp * BLK);
+        *reinterpret_cast<float2*>(base + (gq * TAPS + tap) * TC + cbase) = make_float2(acc[i][0], acc[i][1]);
+        *reinterpret_cast<float2*>(base + ((gq + 8) * TAPS + tap) * TC + cbase) = make_float2(acc[i][2], acc[i][3]);
     }
     __syncthreads();
     float* out = pl.splits == 1 ? dw : partial + (size_t)split * g.k * g.c * R * S;
@@ -150,7 +159,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
     for (int e = threadIdx.x; e < BLK; e += kThreads) {
         float tot = s_red[e];
 #pragma unroll
-        for (int w = 1; w < kWarps; ++w) tot += s_red[w * BLK + e];
+        for (int w = 1; w < SLOTS; ++w) tot += s_red[w * BLK + e];
         const int cc = e % TC, tap = (e / TC) % TAPS, kk = e / (TC * TAPS);
         const int k = k0 + kk, c = c0 + cc;
         if (k < g.k && c < g.c) out[k * g.ws_k + c * g.ws_c + (tap / S) * g.ws_r + (tap % S) * g.ws_s] = scale * tot;
@@ -162,7 +171,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
 bool direct_mma_supported(const Geom& g, const DirectPlan& pl)
 {
     if (g.bf16 || g.xs_c != 1 || g.c % 4 != 0 || g.c < 8) return false;
-    if (g.r != g.s || (g.r != 1 && g.r != 3)) return false;
+    if (g.r != g.s || (g.r != 1 && g.r != 3 && g.r != 5)) return false;
     const int npx = pl.bp * pl.bq, pq = g.p * g.q;
     if (pl.bq != g.q || g.q % 8 != 0 || g.p % pl.bp != 0 || npx % 32 != 0 || npx > 256 || pq % 4 != 0) return false;
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
@@ -188,7 +197,7 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
     const size_t stage = ((size_t)(npx / 32) * 2048 + (size_t)win_h * win_w * TC * 4 + 1023) & ~(size_t)1023;
-    const size_t red = (size_t)kWarps * TK * g.r * g.s * TC * 4;
+    const size_t red = (size_t)(g.r * g.s > 9 ? 1 : kWarps) * TK * g.r * g.s * TC * 4;
     size_t smem = 2 * stage > red ? 2 * stage : red;
     smem += 1024;
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
@@ -203,6 +212,8 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     GACONV_MMA_CASE(1, false)
     GACONV_MMA_CASE(3, true)
     GACONV_MMA_CASE(3, false)
+    GACONV_MMA_CASE(5, true)
+    GACONV_MMA_CASE(5, false)
 #undef GACONV_MMA_CASE
     note_launch();
     if (launch_err != cudaSuccess) return launch_err;

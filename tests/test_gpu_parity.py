@@ -292,6 +292,8 @@ MMA_SHAPES = [
     ConvLayer("mma ragged channels", 3, 24, 16, 16, 20, 3, 3, 1, 1),
     ConvLayer("mma 1x1", 4, 32, 16, 16, 48, 1, 1, 1, 0),
     ConvLayer("mma c8", 7, 8, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("mma 5x5 64->64@16", 3, 64, 16, 16, 64, 5, 5, 1, 2),
+    ConvLayer("mma 5x5 ragged", 4, 20, 16, 16, 24, 5, 5, 1, 2),
 ]
 
 
@@ -313,7 +315,7 @@ def test_fp32_exact_split_tf32_and_fp32_pipes(li):
 
 
 def test_tf32_mode_is_refused_where_it_has_no_kernel():
-    layer = ConvLayer("5x5", 2, 16, 16, 16, 16, 5, 5, 1, 2)
+    layer = ConvLayer("7x7", 2, 16, 16, 16, 16, 7, 7, 1, 3)
     x, dy = _inputs(layer, torch.float32, 320)
     g = GpuLayer(layer, torch.float32, x, dy, math=B.MATH_TF32)
     with pytest.raises(B.GaconvError) as e:
