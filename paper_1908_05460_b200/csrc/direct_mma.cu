@@ -1,6 +1,6 @@
 // Exact filter gradient for fp32 inputs on the warp-level tensor-core path (mma.sync m16n8k8, TF32
 // operands, fp32 accumulate), with the operands split so that fp32 accuracy is kept:
-//   x = big + small,  big = tf32(x),  small = tf32(x - big)
+//   x = big + small,  big = tf32(x) (by truncation),  small = tf32(x - big)
 //   a*b ~= big_a*big_b + big_a*small_b + small_a*big_b            ("3xTF32": error ~ 2^-21 per product)
 // One pass (big*big only) is the opt-in GACONV_MATH_TF32 mode: operands cut to 10 mantissa bits.
 //
@@ -23,11 +23,10 @@ namespace {
 
 constexpr int kThreads = 128, kWarps = 4, TK = 16, TC = 16;
 
-__device__ __forceinline__ uint32_t to_tf32(float v) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
-    return r;
-}
+// TF32 value of v by truncation (the low 13 mantissa bits cleared): one logic op on the full-rate pipe,
+// where cvt.rna.tf32 goes through the conversion unit.  The split stays exact: small = v - big is
+// representable, and its own truncation loses at most 2^-20 of |v|.
+__device__ __forceinline__ uint32_t to_tf32(float v) { return __float_as_uint(v) & 0xffffe000u; }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])

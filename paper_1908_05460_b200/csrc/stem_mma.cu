@@ -35,11 +35,9 @@ struct StemParams {
     int win_h, nt;     // staged rows per item; n-tiles of 8 columns
 };
 
-__device__ __forceinline__ uint32_t to_tf32(float v) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
-    return r;
-}
+// TF32 value of v by truncation (low 13 mantissa bits cleared): one full-rate logic op instead of a trip
+// through the conversion unit; the split x = big + small stays exact.
+__device__ __forceinline__ uint32_t to_tf32(float v) { return __float_as_uint(v) & 0xffffe000u; }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
