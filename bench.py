@@ -413,7 +413,7 @@ def main():
     roof["peak_source"] = peaks["source"]
     # DRAM bytes of one launch from the committed ncu capture of this kernel family (profiles/): the exact
     # fp32 kernel on 16->16@32x32, N=128 moved 16.80 MB for 16.79 MB of algorithmic bytes (no re-reads)
-    roof["traffic"] = {"bytes_per_launch": 16803840, "algorithmic_bytes": 16786432, "layer": "16->16@32 f32 N=128",
+    roof["traffic"] = {"bytes_per_launch": 16800768, "algorithmic_bytes": 16786432, "layer": "16->16@32 f32 N=128",
                        "source": "profiles/direct_mma_f32_16x16_32x32_n128.md"} if roof.get("kernel") == "exact dW" else None
 
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
