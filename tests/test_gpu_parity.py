@@ -349,3 +349,18 @@ def test_stem_layers(li, dtype):
     kcrs = GpuLayer(layer, dtype, x, dy, alpha=2.0, dw_layout=B.DW_KCRS)
     assert norm_err(kcrs.exact(), ref, dn) <= tol(dtype)
     assert B.gaconv_poll_async_status(auto.desc) == B.OK
+
+
+def test_workspace_control_words_are_left_as_found():
+    """Every call must leave the workspace's control block (status word, ticket counters) all zero, so that
+    a workspace initialised once serves any number of calls."""
+    layer = ConvLayer("tickets", 24, 16, 16, 16, 32, 3, 3, 1, 1)
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 500)
+        for algo in (B.ALGO_AUTO, B.ALGO_DIRECT):
+            g = GpuLayer(layer, dtype, x, dy, algo=algo)
+            g.exact(); g.approx(B.METHOD_TOP1); g.approx(B.METHOD_ZERO); g.approx(B.METHOD_RANDOM, seed=3)
+            torch.cuda.synchronize()
+            control = g.ws[:256 + 4096 * 4].cpu()
+            assert int(control.to(torch.int32).abs().sum()) == 0
+            assert B.gaconv_poll_async_status(g.desc) == B.OK
