@@ -44,6 +44,33 @@ reduce_splits_kernel(const V* __restrict__ partial, V* __restrict__ dw, size_t c
     }
 }
 
+// Many splits of a small block (hundreds of 9 KB slots after a small layer): 8 float4 columns per block and
+// 32 split lanes, so that the work spreads over more SMs and every thread has all its loads in flight
+// at once.  Lane l sums splits l, l+32, ... in ascending order; lane 0 of a column adds the 32 subtotals in
+// lane order.
+__global__ void __launch_bounds__(256)
+reduce_splits_many_kernel(const float4* __restrict__ partial, float4* __restrict__ dw, size_t count, int splits, float alpha)
+{
+    __shared__ float4 sm[32][8];
+    pdl_wait_prior_grid();
+    const int cq = threadIdx.x & 7, sl = threadIdx.x >> 3;
+    const size_t i = (size_t)blockIdx.x * 8 + cq;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < count) {
+        const float4* p = partial + i;
+#pragma unroll 8
+        for (int sp = sl; sp < splits; sp += 32) vadd(acc, __ldcg(p + (size_t)sp * count));
+    }
+    sm[sl][cq] = acc;
+    __syncthreads();
+    if (sl == 0 && i < count) {
+        float4 t = sm[0][cq];
+        const int used = splits < 32 ? splits : 32;
+        for (int w = 1; w < used; ++w) vadd(t, sm[w][cq]);
+        dw[i] = vscale(t, alpha);
+    }
+}
+
 }  // namespace
 
 cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int splits, float alpha, cudaStream_t stream)
@@ -52,6 +79,11 @@ cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int spl
     int warps = 1;
     while (warps < splits && warps < kReduceWarps) warps *= 2;
     note_launch();
+    if (count % 4 == 0 && splits >= 64 && count / 4 <= 65536) {
+        const size_t c4 = count / 4;
+        return launch_kernel(reduce_splits_many_kernel, dim3((unsigned)((c4 + 7) / 8)), dim3(256), 0, stream, dim3(1, 1, 1),
+                             reinterpret_cast<const float4*>(partial), reinterpret_cast<float4*>(dw), c4, splits, alpha);
+    }
     if (count % 4 == 0) {
         const size_t c4 = count / 4;
         return launch_kernel(reduce_splits_kernel<float4>, dim3((unsigned)((c4 + 31) / 32)), dim3(32 * warps), 0, stream, dim3(1, 1, 1),
