@@ -133,7 +133,23 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
     }
 }
 
-// four consecutive elements as floats (16-byte load for fp32, 8-byte load for bf16)
+// four consecutive elements, raw (16-byte load for fp32, 8-byte load for bf16), and their values as floats
+struct Raw4 { uint32_t w[4]; };
+__device__ __forceinline__ Raw4 ld4_raw(const float* p) {
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    return Raw4{{t.x, t.y, t.z, t.w}};
+}
+__device__ __forceinline__ Raw4 ld4_raw(const __nv_bfloat16* p) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    return Raw4{{t.x, t.y, 0u, 0u}};
+}
+__device__ __forceinline__ void raw_to_float(const Raw4& r, const float*, float (&v)[4]) {
+    v[0] = __uint_as_float(r.w[0]); v[1] = __uint_as_float(r.w[1]); v[2] = __uint_as_float(r.w[2]); v[3] = __uint_as_float(r.w[3]);
+}
+__device__ __forceinline__ void raw_to_float(const Raw4& r, const __nv_bfloat16*, float (&v)[4]) {
+    v[0] = __uint_as_float(r.w[0] << 16); v[1] = __uint_as_float(r.w[0] & 0xffff0000u);
+    v[2] = __uint_as_float(r.w[1] << 16); v[3] = __uint_as_float(r.w[1] & 0xffff0000u);
+}
 __device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
     const float4 t = __ldg(reinterpret_cast<const float4*>(p));
     v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
@@ -158,7 +174,7 @@ template <> __device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __
 // No global scratch, no atomics; the order of every sum is fixed.
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(512, 2)
-top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x)
+top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x, int NJ)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -169,6 +185,8 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
     int* s_h0 = reinterpret_cast<int*>(s_part + rsc);                   // [ipc] top-left input row of each patch
     int* s_w0 = s_h0 + ipc;
     float* s_sum = reinterpret_cast<float*>(s_w0 + ipc);
+    long long* s_base = reinterpret_cast<long long*>(smem_raw + (((size_t)rsc * 4 + (size_t)ipc * 12 + 7) & ~(size_t)7));   // [ipc] element offset of each patch's top-left pixel
+    float* s_subs = reinterpret_cast<float*>(s_base + ipc);            // [NJ][rsc] lane subtotals
 
     const int k = blockIdx.y, chunk = blockIdx.x, CL = gridDim.x;
     const int n0 = chunk * ipc;
@@ -185,8 +203,9 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
             int best_j; float s;
             scan_map<T, VEC>(dy + ((long long)(n0 + (live ? i : 0)) * g.k + k) * pq, live, pq, G, sub, best_j, s);
             if (live && sub == 0) {
-                s_h0[i] = (best_j / g.q) * g.stride_h - g.pad_h;
-                s_w0[i] = (best_j % g.q) * g.stride_w - g.pad_w;
+                const int h0 = (best_j / g.q) * g.stride_h - g.pad_h, w0 = (best_j % g.q) * g.stride_w - g.pad_w;
+                s_h0[i] = h0; s_w0[i] = w0;
+                s_base[i] = (long long)i * g.xs_n + (long long)h0 * g.xs_h + (long long)w0 * g.xs_w;
                 s_sum[i] = s;
             }
         }
@@ -194,41 +213,46 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
     __syncthreads();
 
     // ---- phase 2: patch accumulate ----
-    // A work item is (element group, image lane j): NJ lanes split the images round-robin
+    // A work item is (element group, image lane j): NJ lanes (chosen by the host: enough that a lane has at
+    // most eight images and that no thread idles) split the images round-robin
     // (i = j, j+NJ, ...), each adding its images in ascending order with up to eight loads in flight;
     // the NJ subtotals are then added in lane order.  VX elements per group: four channels per load
     // on the vector path (NHWC, C a multiple of four), else one.
     {
         const int VX = vec_x ? 4 : 1;
+        constexpr int BATCH = sizeof(T) == 4 ? 4 : 8;          // loads in flight per thread (register budget: 64)
         const int groups = rsc / VX;
-        int NJ = 1;
-        while (NJ * 2 * groups <= (int)blockDim.x && NJ * 2 <= 16) NJ *= 2;
-        float* s_sub = s_part;                                  // NJ == 1: results go straight to s_part
-        if (NJ > 1) s_sub = reinterpret_cast<float*>(s_sum + ipc);   // [NJ][rsc] scratch after the per-image arrays
+        float* s_sub = NJ > 1 ? s_subs : s_part;               // NJ == 1: results go straight to s_part
         for (int item = threadIdx.x; item < groups * NJ; item += blockDim.x) {
             const int j = item / groups, e = (item - j * groups) * VX;
             const int c = e % g.c, rs = e / g.c, s = rs % g.s, r = rs / g.s;
-            const T* xc = x + n0 * g.xs_n + c * g.xs_c;
+            const T* xc = x + n0 * g.xs_n + c * g.xs_c + r * g.xs_h + s * g.xs_w;     // this element of a patch whose corner is pixel (0,0)
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int i0 = j; i0 < cnt; i0 += 8 * NJ) {
-                float v[8][4];
+            for (int i0 = j; i0 < cnt; i0 += BATCH * NJ) {
+                // BATCH loads are issued before any is consumed; they stay raw (two or four registers each)
+                // until then, so that the register allocator has no reason to serialise them
+                Raw4 raw[BATCH];
+                float one[BATCH];
+                bool okv[BATCH];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < BATCH; ++u) {
                     const int i = i0 + u * NJ;
-                    const int hh = (i < cnt ? s_h0[i] : -1) + r, ww = (i < cnt ? s_w0[i] : -1) + s;
-                    const bool ok = i < cnt && hh >= 0 && hh < g.h && ww >= 0 && ww < g.w;
-                    const long long off = ok ? i * g.xs_n + hh * g.xs_h + ww * g.xs_w : 0;   // element 0 is always readable
-                    if (vec_x) ld4(xc + off, v[u]);
-                    else { v[u][0] = ld_as_float(xc + off); v[u][1] = v[u][2] = v[u][3] = 0.f; }
-                    if (!ok) v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+                    const bool in = i < cnt;
+                    okv[u] = in && (unsigned)(s_h0[in ? i : 0] + r) < (unsigned)g.h && (unsigned)(s_w0[in ? i : 0] + s) < (unsigned)g.w;
+                    const T* p = okv[u] ? xc + s_base[i] : x;                           // element 0 is always readable
+                    if (vec_x) raw[u] = ld4_raw(p);
+                    else one[u] = ld_as_float(p);
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < BATCH; ++u) {
                     const int i = i0 + u * NJ;
-                    if (i < cnt) {
+                    if (i < cnt && okv[u]) {
                         const float sm_ = s_sum[i];
+                        float v[4];
+                        if (vec_x) raw_to_float(raw[u], static_cast<const T*>(nullptr), v);
+                        else { v[0] = one[u]; v[1] = v[2] = v[3] = 0.f; }
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) acc[t] = fmaf(sm_, v[u][t], acc[t]);
+                        for (int t = 0; t < 4; ++t) acc[t] = fmaf(sm_, v[t], acc[t]);
                     }
                 }
             }
@@ -393,7 +417,7 @@ cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, f
 bool top1_fused_supported(const Geom& g)
 {
     // the per-channel block of R*S*C sums lives in shared memory
-    return (size_t)g.r * g.s * g.c * sizeof(float) <= 160 * 1024 && g.k <= 65535;
+    return (size_t)g.r * g.s * g.c * sizeof(float) <= 100 * 1024 && g.k <= 65535;
 }
 
 template <typename T, bool VEC>
@@ -406,15 +430,18 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     // 512 threads (two CTAs per SM) where the grid still fits in one wave and the scan would otherwise need
     // two passes over the CTA's maps; measured: helps 32-channel layers, neutral or worse for 16 and 64
     const int threads = (g.k >= 32 && (long long)cl * g.k <= 148 * 2) ? 512 : 256;
-    while (nj * 2 * (rsc / (vec_x ? 4 : 1)) <= threads && nj * 2 <= 16) nj *= 2;
-    const size_t smem = (size_t)rsc * sizeof(float) * (nj > 1 ? 1 + nj : 1) + (size_t)ipc * 12 + 16;
+    const int groups = rsc / (vec_x ? 4 : 1);
+    const int batch = sizeof(T) == 4 ? 4 : 8;
+    while (nj < 16 && (nj * batch < ipc || nj * 2 * groups <= threads)) nj *= 2;    // one batch of images per lane, no idle threads
+    while (nj > 1 && (size_t)rsc * 4 * (1 + nj) > 150 * 1024) nj /= 2;              // the subtotals must fit shared memory
+    const size_t smem = (((size_t)rsc * 4 + (size_t)ipc * 12 + 7) & ~(size_t)7) + (size_t)ipc * 8 + (nj > 1 ? (size_t)nj * rsc * 4 : 0) + 16;
     static size_t configured = 0;
     if (smem > 48 * 1024 && smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(top1_fused_kernel<T, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured = smem;
     }
-    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x);
+    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj);
     note_launch();
     return e;
 }
