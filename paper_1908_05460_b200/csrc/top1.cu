@@ -84,7 +84,14 @@ __device__ __forceinline__ void scan_map(const T* __restrict__ map, bool live, i
             const uint4* mv = reinterpret_cast<const uint4*>(map);
             const int nvec = pq / E;
             int v = sub;
-            // four independent loads in flight per lane before any is consumed
+            // eight, then four independent loads in flight per lane before any is consumed
+            for (; v + 7 * G < nvec; v += 8 * G) {
+                uint4 a[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) a[u] = ld_stream(mv + v + u * G);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) Elem<T>::visit(a[u], (v + u * G) * E, sc);
+            }
             for (; v + 3 * G < nvec; v += 4 * G) {
                 uint4 a = ld_stream(mv + v), b = ld_stream(mv + v + G), c = ld_stream(mv + v + 2 * G),
                       d = ld_stream(mv + v + 3 * G);
@@ -441,6 +448,8 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
         if (e != cudaSuccess) return e;
         configured = smem;
     }
+    // lanes per map: few enough that one pass covers all the CTA's maps (their loads are then all in flight at once)
+    while (G > 1 && G * ipc > threads) G /= 2;
     cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj);
     note_launch();
     return e;
