@@ -15,27 +15,11 @@
 // fixed order) and the CTA writes its block: to dW if it is the only split, else to its slot of
 // the partial buffer, which reduce_splits() adds up in split order.
 #include "gaconv_internal.h"
+#include "device_utils.cuh"
 #include "tma.cuh"
 
 namespace gaconv {
 namespace {
-
-template <typename T> __device__ __forceinline__ float ldf(const T* p);
-template <> __device__ __forceinline__ float ldf<float>(const float* p) { return __ldg(p); }
-template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) {
-    return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
-}
-
-// four consecutive elements as floats (16-byte load for fp32, 8-byte load for bf16)
-__device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
-    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
-    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-}
-__device__ __forceinline__ void ld4(const __nv_bfloat16* p, float (&v)[4]) {
-    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
-    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
-}
 
 constexpr int kThreads = 128;
 

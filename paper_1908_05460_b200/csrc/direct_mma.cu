@@ -16,6 +16,7 @@
 //   dY box: 32 pixels x 16 channels with the 128-byte TMA swizzle, so that the eight k-rows a fragment
 //   load touches fall in different banks.
 #include "gaconv_internal.h"
+#include "device_utils.cuh"
 #include "tma.cuh"
 
 namespace gaconv {
@@ -23,15 +24,6 @@ namespace {
 
 constexpr int kThreads = 128, kWarps = 4, TK = 16, TC = 16;
 
-// TF32 value of v by truncation (the low 13 mantissa bits cleared): one logic op on the full-rate pipe,
-// where cvt.rna.tf32 goes through the conversion unit.  The split stays exact: small = v - big is
-// representable, and its own truncation loses at most 2^-20 of |v|.
-__device__ __forceinline__ uint32_t to_tf32(float v) { return __float_as_uint(v) & 0xffffe000u; }
-__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
 template <int R, int S, bool THREE_PASS>
 __global__ void __launch_bounds__(kThreads)

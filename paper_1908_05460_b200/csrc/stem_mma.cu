@@ -17,6 +17,7 @@
 #include <cstring>
 
 #include "gaconv_internal.h"
+#include "device_utils.cuh"
 #include "tma.cuh"
 
 namespace gaconv {
@@ -35,19 +36,6 @@ struct StemParams {
     int win_h, nt;     // staged rows per item; n-tiles of 8 columns
 };
 
-// TF32 value of v by truncation (low 13 mantissa bits cleared): one full-rate logic op instead of a trip
-// through the conversion unit; the split x = big + small stays exact.
-__device__ __forceinline__ uint32_t to_tf32(float v) { return __float_as_uint(v) & 0xffffe000u; }
-__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
 template <typename T, int NT>
 __global__ void __launch_bounds__(kThreads)

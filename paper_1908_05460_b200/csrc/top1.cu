@@ -10,6 +10,7 @@
 #include <cooperative_groups.h>
 
 #include "gaconv_internal.h"
+#include "device_utils.cuh"
 
 namespace gaconv {
 
@@ -157,20 +158,6 @@ __device__ __forceinline__ void raw_to_float(const Raw4& r, const __nv_bfloat16*
     v[0] = __uint_as_float(r.w[0] << 16); v[1] = __uint_as_float(r.w[0] & 0xffff0000u);
     v[2] = __uint_as_float(r.w[1] << 16); v[3] = __uint_as_float(r.w[1] & 0xffff0000u);
 }
-__device__ __forceinline__ void ld4(const float* p, float (&v)[4]) {
-    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
-    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-}
-__device__ __forceinline__ void ld4(const __nv_bfloat16* p, float (&v)[4]) {
-    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
-    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
-}
-template <typename T> __device__ __forceinline__ float ld_as_float(const T* p);
-template <> __device__ __forceinline__ float ld_as_float<float>(const float* p) { return __ldg(p); }
-template <> __device__ __forceinline__ float ld_as_float<__nv_bfloat16>(const __nv_bfloat16* p) {
-    return bf16_bits_to_float(__ldg(reinterpret_cast<const unsigned short*>(p)));
-}
 
 // Algorithm 1 in one launch.  grid (CL, K), thread-block clusters of CL CTAs along x: the CL CTAs of
 // a cluster share one output channel k and split the batch into CL contiguous ranges of images.
@@ -248,7 +235,7 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
                     okv[u] = in && (unsigned)(s_h0[in ? i : 0] + r) < (unsigned)g.h && (unsigned)(s_w0[in ? i : 0] + s) < (unsigned)g.w;
                     const T* p = okv[u] ? xc + s_base[i] : x;                           // element 0 is always readable
                     if (vec_x) raw[u] = ld4_raw(p);
-                    else one[u] = ld_as_float(p);
+                    else one[u] = ldf(p);
                 }
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
@@ -329,7 +316,7 @@ gather_kernel(const T* __restrict__ x, const int32_t* __restrict__ idx, const fl
         for (int i = 0; i < cnt; ++i) {
             const int hh = s_h0[i] + r, ww = s_w0[i] + s;
             if (hh >= 0 && hh < g.h && ww >= 0 && ww < g.w)
-                acc = fmaf(s_sum[i], ld_as_float(x + (n0 + i) * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w), acc);
+                acc = fmaf(s_sum[i], ldf(x + (n0 + i) * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w), acc);
         }
         if (chunks == 1) dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * acc;
         else part[e] = acc;
