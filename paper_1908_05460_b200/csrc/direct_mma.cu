@@ -1,8 +1,10 @@
-// Exact filter gradient for fp32 inputs on the warp-level tensor-core path (mma.sync m16n8k8, TF32
-// operands, fp32 accumulate), with the operands split so that fp32 accuracy is kept:
+// Exact filter gradient on the warp-level tensor-core path.  fp32 inputs (the main use): mma.sync m16n8k8,
+// TF32 operands, fp32 accumulate, with the operands split so that fp32 accuracy is kept:
 //   x = big + small,  big = tf32(x) (by truncation),  small = tf32(x - big)
 //   a*b ~= big_a*big_b + big_a*small_b + small_a*big_b            ("3xTF32": error ~ 2^-21 per product)
 // One pass (big*big only) is the opt-in GACONV_MATH_TF32 mode: operands cut to 10 mantissa bits.
+// bf16 inputs run one pass of m16n8k16; the tcgen05 kernel is faster wherever it tiles the shape (measured
+// 11-12 us against 13-14 us on the 16- and 32-channel ResNet-20 layers), so this serves the remaining shapes.
 //
 //   dW[k,c,r,s] = alpha * sum_{n,p,q} Xz[n,c,p*st+r-pad,q*st+s-pad] * dY[n,k,p,q]              (Section 2.4)
 //
@@ -25,7 +27,8 @@ namespace {
 constexpr int kThreads = 128, kWarps = 4, TK = 16, TC = 16;
 
 
-template <int R, int S, bool THREE_PASS>
+// BF16: bf16 inputs on m16n8k16 (one pass, products exact in fp32; 64 pixels per dY box, 16 per k-step).
+template <int R, int S, bool THREE_PASS, bool BF16>
 __global__ void __launch_bounds__(kThreads)
 direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ status,
                   const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
@@ -44,8 +47,9 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
 
     const int npx = pl.bp * pl.bq;                       // a multiple of 32; bq == Q, a multiple of 8
     const int win_h = (pl.bp - 1) * g.stride_h + R, win_w = (pl.bq - 1) * g.stride_w + S;
-    const int dy_bytes = npx / 32 * 2048;                // [npx/32 boxes][16 k][32 px], 128-byte swizzled rows
-    const int x_bytes = win_h * win_w * TC * 4;          // [row][col][16 c]
+    constexpr int EB = BF16 ? 2 : 4, BOXPX = BF16 ? 64 : 32, KPX = BF16 ? 16 : 8;
+    const int dy_bytes = npx / BOXPX * 2048;             // [boxes][16 k][128-byte swizzled rows]
+    const int x_bytes = win_h * win_w * TC * EB;         // [row][col][16 c]
     const int stage_bytes = (dy_bytes + x_bytes + 1023) & ~1023;
     uint8_t* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
 
@@ -65,7 +69,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
         const uint32_t full = smem_u32(&bar_full[stage]);
         const uint32_t dst = smem_u32(smem + stage * stage_bytes);
         mbar_expect_tx(full, (uint32_t)(dy_bytes + x_bytes));
-        for (int b = 0; b < npx / 32; ++b) tma_load_3d(dst + b * 2048, &map_dy, full, p0 * g.q + 32 * b, k0, n);
+        for (int b = 0; b < npx / BOXPX; ++b) tma_load_3d(dst + b * 2048, &map_dy, full, p0 * g.q + BOXPX * b, k0, n);
         tma_load_4d(dst + dy_bytes, &map_x, full, c0, -g.pad_w, p0 * g.stride_h - g.pad_h, n);
     };
     if (threadIdx.x == 0) {
@@ -87,10 +91,38 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
         __syncthreads();
         if (s_fail) { if (threadIdx.x == 0) atomicOr(status, 1u); break; }   // uniform exit
         const uint8_t* s_dy = smem + stage * stage_bytes;
-        const float* s_x = reinterpret_cast<const float*>(s_dy + dy_bytes);
+        const float* s_x = reinterpret_cast<const float*>(s_dy + dy_bytes);   // bf16 inputs: reinterpreted below
 
-        for (int ks = SPLIT_TAPS ? 0 : warp; ks < npx / 8; ks += SPLIT_TAPS ? 1 : kWarps) {
-            const int px0 = ks * 8;
+        for (int ks = SPLIT_TAPS ? 0 : warp; ks < npx / KPX; ks += SPLIT_TAPS ? 1 : kWarps) {
+            const int px0 = ks * KPX;
+            if constexpr (BF16) {
+                // A: dY[k = gq (+8)][px0 + 2*tq, +1 (+8, +9)], two bf16 per register
+                uint32_t a[4];
+                const uint8_t* box = s_dy + (px0 >> 6) * 2048;
+                const int ch0 = (px0 & 63) >> 3;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = gq + (i & 1) * 8, ch = ch0 + (i >> 1);
+                    a[i] = *reinterpret_cast<const uint32_t*>(box + row * 128 + ((ch ^ (row & 7)) << 4) + tq * 4);
+                }
+                const int pp = px0 / pl.bq, qq = px0 - pp * pl.bq;
+                const unsigned short* xrow = reinterpret_cast<const unsigned short*>(s_x) + ((pp * g.stride_h) * win_w + (qq + 2 * tq) * g.stride_w) * TC + gq;
+                const int px1 = g.stride_w * TC, px8 = 8 * px1;
+#pragma unroll
+                for (int i = 0; i < TPW; ++i) {
+                    const int tap = tap_lo + i;
+                    if (SPLIT_TAPS && tap >= TAPS) break;
+                    const int r = SPLIT_TAPS ? tap / S : i / S, s = SPLIT_TAPS ? tap % S : i % S;
+                    const unsigned short* xt = xrow + (r * win_w + s) * TC;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t b0 = (uint32_t)xt[h * 8] | ((uint32_t)xt[h * 8 + px1] << 16);
+                        const uint32_t b1 = (uint32_t)xt[h * 8 + px8] | ((uint32_t)xt[h * 8 + px8 + px1] << 16);
+                        mma_bf16(acc[i * 2 + h], a, b0, b1);
+                    }
+                }
+                continue;
+            }
             // ---- A fragment: dY[k = gq (+8)][px0 + tq (+4)], from the swizzled box ----
             uint32_t a_big[4], a_small[4];
             {
@@ -161,10 +193,11 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
 
 bool direct_mma_supported(const Geom& g, const DirectPlan& pl)
 {
-    if (g.bf16 || g.xs_c != 1 || g.c % 4 != 0 || g.c < 8) return false;
+    if (g.xs_c != 1 || g.c % (g.bf16 ? 8 : 4) != 0 || g.c < 8) return false;
     if (g.r != g.s || (g.r != 1 && g.r != 3 && g.r != 5)) return false;
     const int npx = pl.bp * pl.bq, pq = g.p * g.q;
-    if (pl.bq != g.q || g.q % 8 != 0 || g.p % pl.bp != 0 || npx % 32 != 0 || npx > 256 || pq % 4 != 0) return false;
+    const int boxpx = g.bf16 ? 64 : 32, kpx = g.bf16 ? 16 : 8;
+    if (pl.bq != g.q || g.q % kpx != 0 || g.p % pl.bp != 0 || npx % boxpx != 0 || npx > 256 || pq % 8 != 0) return false;
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
     if (win_h > 256 || win_w > 256) return false;
     return encode_fn() != nullptr;
@@ -177,25 +210,27 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
     CUtensorMap map_dy, map_x;
     cuuint64_t d3[3] = {(cuuint64_t)pq, (cuuint64_t)g.k, (cuuint64_t)g.n};
-    cuuint64_t s3[2] = {(cuuint64_t)pq * 4, (cuuint64_t)g.k * pq * 4};
-    cuuint32_t b3[3] = {32, (cuuint32_t)TK, 1}, e3[3] = {1, 1, 1};
+    const int eb = g.bf16 ? 2 : 4, boxpx = g.bf16 ? 64 : 32;
+    const CUtensorMapDataType dt = g.bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    cuuint64_t s3[2] = {(cuuint64_t)pq * eb, (cuuint64_t)g.k * pq * eb};
+    cuuint32_t b3[3] = {(cuuint32_t)boxpx, (cuuint32_t)TK, 1}, e3[3] = {1, 1, 1};
     cuuint64_t d4[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
-    cuuint64_t s4[3] = {(cuuint64_t)g.c * 4, (cuuint64_t)g.w * g.c * 4, (cuuint64_t)g.h * g.w * g.c * 4};
+    cuuint64_t s4[3] = {(cuuint64_t)g.c * eb, (cuuint64_t)g.w * g.c * eb, (cuuint64_t)g.h * g.w * g.c * eb};
     cuuint32_t b4[4] = {(cuuint32_t)TC, (cuuint32_t)win_w, (cuuint32_t)win_h, 1}, e4[4] = {1, 1, 1, 1};
-    if (encode_fn()(&map_dy, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(dy), d3, s3, b3, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    if (encode_fn()(&map_dy, dt, 3, const_cast<void*>(dy), d3, s3, b3, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
-        encode_fn()(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(x), d4, s4, b4, e4, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        encode_fn()(&map_x, dt, 4, const_cast<void*>(x), d4, s4, b4, e4, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    const size_t stage = ((size_t)(npx / 32) * 2048 + (size_t)win_h * win_w * TC * 4 + 1023) & ~(size_t)1023;
+    const size_t stage = ((size_t)(npx / boxpx) * 2048 + (size_t)win_h * win_w * TC * eb + 1023) & ~(size_t)1023;
     const size_t red = (size_t)(g.r * g.s > 9 ? 1 : kWarps) * TK * g.r * g.s * TC * 4;
     size_t smem = 2 * stage > red ? 2 * stage : red;
     smem += 1024;
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
     cudaError_t launch_err = cudaErrorInvalidValue;
 #define GACONV_MMA_CASE(RR, TP)                                                                                          \
-    if (g.r == RR && three_pass == TP) {                                                                                 \
-        auto kern = direct_mma_kernel<RR, RR, TP>;                                                                       \
+    if (g.r == RR && three_pass == TP && !g.bf16) {                                                                      \
+        auto kern = direct_mma_kernel<RR, RR, TP, false>;                                                                       \
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
         launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), dw, partial, status, map_dy, map_x, g, pl); \
     }
@@ -206,6 +241,16 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     GACONV_MMA_CASE(5, true)
     GACONV_MMA_CASE(5, false)
 #undef GACONV_MMA_CASE
+#define GACONV_MMA_BF16_CASE(RR)                                                                                         \
+    if (g.r == RR && g.bf16) {                                                                                           \
+        auto kern = direct_mma_kernel<RR, RR, false, true>;                                                             \
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+        launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), dw, partial, status, map_dy, map_x, g, pl); \
+    }
+    GACONV_MMA_BF16_CASE(1)
+    GACONV_MMA_BF16_CASE(3)
+    GACONV_MMA_BF16_CASE(5)
+#undef GACONV_MMA_BF16_CASE
     note_launch();
     if (launch_err != cudaSuccess) return launch_err;
     if (pl.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.c * g.r * g.s, pl.splits, g.alpha, stream);
