@@ -364,3 +364,38 @@ def test_workspace_control_words_are_left_as_found():
             control = g.ws[:256 + 4096 * 4].cpu()
             assert int(control.to(torch.int32).abs().sum()) == 0
             assert B.gaconv_poll_async_status(g.desc) == B.OK
+
+
+def _fuzz_shapes():
+    rng = np.random.default_rng(20261125)
+    out = []
+    while len(out) < 28:
+        r = int(rng.choice([1, 3, 5]))
+        hw = int(rng.choice([2, 4, 7, 8, 16, 32]))
+        stride = int(rng.choice([1, 2]))
+        pad = int(rng.choice([0, r // 2]))
+        if hw + 2 * pad < r:
+            continue
+        out.append(ConvLayer("fuzz%d" % len(out), int(rng.integers(1, 7)), int(rng.choice([1, 3, 8, 16, 24, 32, 64, 72])),
+                             hw, hw, int(rng.choice([1, 8, 16, 24, 64, 80, 128])), r, r, stride, pad, dy_std=1.0))
+    return out
+
+
+FUZZ = _fuzz_shapes()
+
+
+@pytest.mark.parametrize("li", range(len(FUZZ)), ids=["%s c%d k%d hw%d r%d s%d p%d" % (l.name, l.c, l.k, l.h, l.r, l.stride, l.pad) for l in FUZZ])
+def test_seeded_random_geometries(li):
+    """Planner robustness: whatever kernel a geometry is routed to, exact dW and top-1 match the oracle."""
+    layer = FUZZ[li]
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 600 + li)
+        xd, dyd = to_f64(x), to_f64(dy)
+        g = GpuLayer(layer, dtype, x, dy)
+        ref, dn = oracle.dw_exact(xd, dyd, oshape(layer))
+        assert norm_err(g.exact(), ref, dn) <= tol(dtype)
+        idx, _, _ = g.select()
+        np.testing.assert_array_equal(idx, oracle.top1_select(dyd)[0])
+        ref, dn = oracle.dw_top1(xd, dyd, oshape(layer))
+        assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
+        assert B.gaconv_poll_async_status(g.desc) == B.OK
