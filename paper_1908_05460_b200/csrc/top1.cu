@@ -137,7 +137,15 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
     if (sub == 0) { idx[m] = best_j; sum[m] = s; }
     if (dy_sparse != nullptr) {
         T* out = dy_sparse + m * (long long)pq;
-        for (int j = sub; j < pq; j += G) Elem<T>::store1(out + j, j == best_j ? s : 0.0f);
+        if (VEC) {      // 16-byte zero vectors, then the one retained entry
+            constexpr int E = Elem<T>::kPerVec;
+            uint4* ov = reinterpret_cast<uint4*>(out);
+            for (int v = sub; v < pq / E; v += G) ov[v] = make_uint4(0u, 0u, 0u, 0u);
+            __syncwarp();
+            if (sub == 0) Elem<T>::store1(out + best_j, s);
+        } else {
+            for (int j = sub; j < pq; j += G) Elem<T>::store1(out + j, j == best_j ? s : 0.0f);
+        }
     }
 }
 
