@@ -15,11 +15,15 @@
 //        the 32 lanes of each TMEM sub-partition, so two accumulators share the same columns.
 // A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks.  Consecutive
 // splits form a thread-block cluster and add their blocks through distributed shared memory; if a tile
-// has several clusters, a second, element-parallel kernel adds the clusters' slots in order.
+// has several clusters, each cluster leaves its sum in a slot of the workspace and the last cluster of
+// the tile to finish a slice adds the slots of that slice in slot order (a ticket per slice), so the
+// order of every sum is fixed whatever the timing.
 //
 // Warp roles: warp 0 = TMA producer; warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns
 // the TMEM allocation); warps 4..7 = epilogue.  The filter rows are dealt round-robin to the issuers:
-// a single thread sustains only one small MMA per ~60 cycles, and rows accumulate independently.
+// a single thread sustains only one small MMA per ~60-100 cycles, and rows accumulate independently.
+// A CTA that holds a single filter row keeps TWO accumulators for it: two issuers take alternate chunks
+// of the reduction, and the epilogue adds accumulator 0 + accumulator 1 (a fixed order).
 // Every mbarrier wait is bounded; on expiry the kernel raises the workspace status word, drains
 // the copies it has in flight, frees its tensor memory and returns.
 #include <cuda.h>
@@ -31,6 +35,14 @@
 
 #include "gaconv_internal.h"
 #include "tma.cuh"
+
+// GACONV_TUNING builds carry clock64 stamps of CTA (0,0)'s phases (workspace bytes [64,128)) and read
+// planner overrides from the environment; the default build has neither.
+#ifdef GACONV_TUNING
+#define GACONV_TL(slot, cond) do { if (tl && (cond)) tl[slot] = clock64(); } while (0)
+#else
+#define GACONV_TL(slot, cond) do { } while (0)
+#endif
 
 namespace gaconv {
 namespace {
@@ -67,12 +79,15 @@ struct TcParams {
     int m;              // MMA M: 64 or 128 output channels per k-tile
     int kb;             // rows of an A box (k rounded up to 8, at most m)
     int ct;             // input channels per c-tile; MMA N = s * ct
+    int ct_shift;       // log2(ct)
     int tiles_k, tiles_c, splits;
+    int chunk_base, chunk_rem;   // split i takes chunk_base chunks, one more when i < chunk_rem
     int halo;           // 1: S tiles with R-1 halo rows, row shift = row offset; 0: R*S tiles
-    int ci, bp;         // chunk = ci images x bp output rows (ci > 1 only when the map has < 64 pixels)
+    int ci, bp;         // chunk = ci images x bp output rows (ci > 1: whole maps)
     int chunks;         // total chunks of the reduction
     int a_sub_px;       // pixels per A box = min(64, PQ)
     int a_subs;         // A boxes per chunk
+    int a_subs_img;     // A boxes per image of a chunk (maps of 64 pixels and more)
     int a_sub_bytes;    // kb * a_sub_px * 2
     int a_region_bytes; // a_subs * a_sub_bytes rounded up to 1 KiB (B tiles start there)
     int a_swz, b_swz;   // swizzle codes of the descriptors
@@ -89,12 +104,14 @@ struct TcParams {
     int stage_bytes, stages;
     int ksteps;         // ci*bp*Q/16
     int tmem_cols;      // power of two >= 32
-    int cl;             // thread-block cluster size along the split dimension (1, 2, 4 or 8); divides splits
-    int rsplit;         // 1: a CTA handles ONE filter row (tile index carries r); M = 128, N = s * 64
+    int cl;             // thread-block cluster size along the split dimension (1..4); divides splits
+    int rsplit;         // 1: a CTA handles ONE filter row (tile index carries r); N = s * 64
     int rc;             // filter rows per CTA: g.r, or 1 when rsplit
-    int issuers;        // MMA-issuing warps: min(R, 3); issuer i takes filter rows i, i+issuers, ...
+    int dual;           // 1 (only with rc == 1): two accumulators, issuer i takes the chunks with (index & 1) == i
+    int issuers;        // MMA-issuing warps: min(R, 3), or 2 when dual; issuer i takes filter rows i, i+issuers, ...
+    int slot_quads;     // float4 elements of one cluster slot (m rows x rc * s * ct columns)
     uint32_t idesc;
-    int timeline;       // 1: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
+    int timeline;       // tuning builds: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
 };
 
 constexpr int kMaxStages = 8;
@@ -111,6 +128,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
+    __shared__ int s_last;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -120,16 +138,18 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int r_lo = P.rsplit ? tile % g.r : 0;                 // first filter row of this CTA
     const int kc_tile = P.rsplit ? tile / g.r : tile;
     const int k0 = (kc_tile / P.tiles_c) * P.m, c0 = (kc_tile % P.tiles_c) * P.ct;
-    const int per = (P.chunks + P.splits - 1) / P.splits;
-    const int ch_begin = min(P.chunks, split * per), ch_end = min(P.chunks, ch_begin + per);
-    const int nchunks = ch_end - ch_begin;
+    const int ch_begin = split * P.chunk_base + min(split, P.chunk_rem);
+    const int nchunks = P.chunk_base + (split < P.chunk_rem ? 1 : 0);
     const int nmma = g.s * P.ct;
     float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // reduction block, aliases the stages
     const int red_stride = P.rc * nmma + 4;
 
     pdl_release_next_grid();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), P.issuers); }
+        // the tensor maps are kernel parameters: fetching them does not depend on the previous kernel
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_dy) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        for (int i = 0; i < P.stages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), P.dual ? 1 : P.issuers); }
         mbar_init(smem_u32(&bar_acc), P.issuers);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -143,14 +163,16 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = s_tmem_base;
     pdl_wait_prior_grid();     // set-up done; from here on global memory of the previous kernel is read and written
+#ifdef GACONV_TUNING
     long long* tl = (P.timeline && blockIdx.x == 0 && blockIdx.y == 0) ? reinterpret_cast<long long*>(status + 16) : nullptr;
-    if (tl && threadIdx.x == 0) tl[0] = clock64();
+#endif
+    GACONV_TL(0, threadIdx.x == 0);
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer
         // chunk coordinates advance incrementally: no division inside the loop
         int n0, p0;
-        const bool whole_maps = P.by_image != 0;
+        const bool whole_maps = P.by_image != 0 || P.ci > 1;
         const int cpi = whole_maps ? 1 : g.p / P.bp;
         if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
@@ -165,11 +187,14 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             mbar_expect_tx(full, tx_bytes);
             if (P.tiny) {                                                        // one box per 64-channel atom
                 for (int a = 0; a * 64 < P.m; ++a) tma_load_3d(sa + a * P.a_lbo, &map_dy, full, k0 + 64 * a, 0, n0);
-            } else if (whole_maps) {
+            } else if (P.by_image) {
                 tma_load_3d(sa, &map_dy, full, 0, k0, n0);                       // ci whole maps in one box
             } else {
-                int px = p0 * g.q;
-                for (int b = 0; b < P.a_subs; ++b, px += 64) tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, px, k0, n0);
+                uint32_t dst = sa;                                               // images past the batch read as zeros
+                for (int i = 0; i < P.ci; ++i) {
+                    int px = p0 * g.q;
+                    for (int b = 0; b < P.a_subs_img; ++b, px += 64, dst += P.a_sub_bytes) tma_load_3d(dst, &map_dy, full, px, k0, n0 + i);
+                }
             }
             if (P.wide) {
                 tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
@@ -217,45 +242,48 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         int nrows = 0;
 #pragma unroll
         for (int i = 0; i < RI; ++i) {
-            const int r = issuer + i * P.issuers;
+            const int r = issuer + i * P.issuers;                   // dual: accumulator index, both on filter row 0 of the CTA
             d_row[i] = P.m == 128 ? tmem_base + r * nmma : tmem_base + (((uint32_t)(r & 1) * 16u) << 16) + (r >> 1) * nmma;
-            b_row[i] = r * b_r_step;
-            if (r < R) nrows = i + 1;
+            b_row[i] = P.dual ? 0u : r * b_r_step;
+            if (P.dual ? i == 0 : r < R) nrows = i + 1;
         }
         const uint64_t a_hi64 = (uint64_t)a_hi << 32, b_hi64 = (uint64_t)b_hi << 32;
         const uint32_t idesc = P.idesc;
+        const int mine = P.dual ? issuer : 0, it_step_mask = P.dual ? 1 : 0;
         int st = 0, ph = 0;
         bool fresh = true;            // the next k-step starts the accumulation (overwrites TMEM)
         for (int it = 0; it < nchunks; ++it) {
-            if (!mbar_wait(smem_u32(&bar_full[st]), ph)) { s_abort = 1; atomicOr(status, 1u); break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (tl && it == 0 && issuer == 0) tl[1] = clock64();
-            const uint32_t sa = smem_base + st * P.stage_bytes;
-            // 14-bit start-address fields: in a cluster launch shared addresses carry the CTA rank in high bits
-            uint32_t a_lo = a_lo_c | ((sa >> 4) & 0x3fffu);
-            uint32_t b_lo = b_lo_c | (((sa + P.a_region_bytes) >> 4) & 0x3fffu);
-            for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
-                if (fresh) {      // first k-step of this CTA: accumulate flag off
-#pragma unroll
-                    for (int i = 0; i < RI; ++i)
-                        if (i < nrows) umma_bf16(d_row[i], a_hi64 | a_lo, b_hi64 | (b_lo + b_row[i]), idesc, 0u);
-                }
-#pragma unroll
-                for (int k4 = 0; k4 < KS; ++k4) {
-                    if (!(fresh && k4 == 0)) {
+            if ((it & it_step_mask) == mine) {
+                if (!mbar_wait(smem_u32(&bar_full[st]), ph)) { s_abort = 1; atomicOr(status, 1u); break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                GACONV_TL(1, it == 0 && issuer == 0);
+                const uint32_t sa = smem_base + st * P.stage_bytes;
+                // 14-bit start-address fields: in a cluster launch shared addresses carry the CTA rank in high bits
+                uint32_t a_lo = a_lo_c | ((sa >> 4) & 0x3fffu);
+                uint32_t b_lo = b_lo_c | (((sa + P.a_region_bytes) >> 4) & 0x3fffu);
+                for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
+                    if (fresh) {      // first k-step of this accumulator: accumulate flag off
 #pragma unroll
                         for (int i = 0; i < RI; ++i)
-                            if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + a_k4 * k4), b_hi64 | (b_lo + b_k_off[k4] + b_row[i]), idesc);
+                            if (i < nrows) umma_bf16(d_row[i], a_hi64 | a_lo, b_hi64 | (b_lo + b_row[i]), idesc, 0u);
                     }
+#pragma unroll
+                    for (int k4 = 0; k4 < KS; ++k4) {
+                        if (!(fresh && k4 == 0)) {
+#pragma unroll
+                            for (int i = 0; i < RI; ++i)
+                                if (i < nrows) umma_bf16_acc(d_row[i], a_hi64 | (a_lo + a_k4 * k4), b_hi64 | (b_lo + b_k_off[k4] + b_row[i]), idesc);
+                        }
+                    }
+                    fresh = false;
+                    b_lo += b_sub_step;
                 }
-                fresh = false;
-                b_lo += b_sub_step;
+                umma_commit(smem_u32(&bar_empty[st]));   // frees the stage once these MMAs have read it
             }
-            umma_commit(smem_u32(&bar_empty[st]));   // frees the stage once these MMAs have read it
             if (++st == P.stages) { st = 0; ph ^= 1; }
         }
         umma_commit(smem_u32(&bar_acc));             // accumulators complete
-        if (tl && issuer == 0) tl[2] = clock64();
+        GACONV_TL(2, issuer == 0);
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue 1: TMEM -> shared memory
         // The accumulators go to a [row][column] fp32 block in this CTA's shared memory (the operand
@@ -264,39 +292,75 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const bool ready = mbar_wait_sleepy(smem_u32(&bar_acc), 0);
         if (!ready) { s_abort = 1; atomicOr(status, 1u); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (tl && threadIdx.x == 128) tl[3] = clock64();
+        GACONV_TL(3, threadIdx.x == 128);
         if (ready && !s_abort) {
             const int sp = warp & 3;
-            const int groups = P.m == 128 ? P.rc : (P.rc + 1) / 2;
-            const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
-            for (int gi = 0; gi < groups; ++gi) {
-                const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's filter rows
-                const bool row_ok = rl < P.rc && k0 + row < g.k;
-                const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
-                float* rrow = red + row * red_stride + rl * nmma;
-                for (int col = 0; col < nmma; col += 64) {
-                    float v[4][16];                                        // up to four 16-column loads in flight
-                    const int nld = min(4, (nmma - col) >> 4);
+            if (P.dual) {
+                // accumulator 0 (even chunks) + accumulator 1 (odd chunks).  M = 128: they sit side by side in the
+                // columns; M = 64: in the two 16-lane halves of each sub-partition (lane l and lane l + 16).
+                const bool has0 = nchunks > 0, has1 = nchunks > 1;
+                const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
+                const bool row_ok = k0 + row < g.k && (P.m == 128 || lane < 16);
+                const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16);
+                float* rrow = red + row * red_stride;
+                for (int col = 0; col < nmma; col += 32) {
+                    float v0[2][16], v1[2][16];
+                    const int nld = min(2, (nmma - col) >> 4);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (u < nld) tmem_ld16_nowait(tbase + col + 16 * u, v[u]);
+                    for (int u = 0; u < 2; ++u)
+                        if (u < nld) {
+                            tmem_ld16_nowait(tbase + col + 16 * u, v0[u]);
+                            if (P.m == 128) tmem_ld16_nowait(tbase + nmma + col + 16 * u, v1[u]);
+                        }
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (!row_ok) continue;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 2; ++u) {
                         if (u >= nld) continue;
+                        float t[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float a0 = v0[u][e];
+                            const float a1 = P.m == 128 ? v1[u][e] : __shfl_down_sync(0xffffffffu, a0, 16);
+                            t[e] = (has0 ? a0 : 0.f) + (has1 ? a1 : 0.f);
+                        }
+                        if (!row_ok) continue;
                         float4* p4 = reinterpret_cast<float4*>(rrow + col + 16 * u);
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4)
-                            p4[q4] = nchunks > 0 ? make_float4(v[u][4 * q4], v[u][4 * q4 + 1], v[u][4 * q4 + 2], v[u][4 * q4 + 3])
-                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int q4 = 0; q4 < 4; ++q4) p4[q4] = make_float4(t[4 * q4], t[4 * q4 + 1], t[4 * q4 + 2], t[4 * q4 + 3]);
+                    }
+                }
+            } else {
+                const int groups = P.m == 128 ? P.rc : (P.rc + 1) / 2;
+                const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
+                for (int gi = 0; gi < groups; ++gi) {
+                    const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's filter rows
+                    const bool row_ok = rl < P.rc && k0 + row < g.k;
+                    const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
+                    float* rrow = red + row * red_stride + rl * nmma;
+                    for (int col = 0; col < nmma; col += 64) {
+                        float v[4][16];                                        // up to four 16-column loads in flight
+                        const int nld = min(4, (nmma - col) >> 4);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (u < nld) tmem_ld16_nowait(tbase + col + 16 * u, v[u]);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (!row_ok) continue;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (u >= nld) continue;
+                            float4* p4 = reinterpret_cast<float4*>(rrow + col + 16 * u);
+#pragma unroll
+                            for (int q4 = 0; q4 < 4; ++q4)
+                                p4[q4] = nchunks > 0 ? make_float4(v[u][4 * q4], v[u][4 * q4 + 1], v[u][4 * q4 + 2], v[u][4 * q4 + 3])
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
                     }
                 }
             }
         }
     }
 
-    if (tl && threadIdx.x == 128) tl[4] = clock64();
+    GACONV_TL(4, threadIdx.x == 128);
     // ---------------------------------------------------------------------- TMEM teardown
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -309,34 +373,45 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     // The cl CTAs of a cluster are consecutive splits of one output tile.  After a cluster barrier CTA
     // `rank` adds slice `rank` of the block over the cl CTAs through distributed shared memory, in
     // rank order.  With one cluster per tile the result (times alpha) goes straight to dW; with several,
-    // to the cluster's slot of the partial buffer, which reduce_splits() adds up in slot order afterwards.
-    // A CTA that gave up on a wait still takes part in the barriers, so its peers never wait in vain.
+    // to the cluster's slot in the workspace, and the last cluster of the tile to deliver slice `rank`
+    // (a ticket per tile and slice) adds that slice over the slots in slot order and writes dW.
+    // A CTA that gave up on a wait still takes part in the barriers and the ticket, so its peers never
+    // wait in vain and the counters return to zero.
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     const int cl = P.cl, rank = cl > 1 ? (int)cluster.block_rank() : 0;
     const int groups_per_tile = P.splits / cl, cgroup = split / cl;
     if (cl > 1) cluster.sync();
-    if (tl && threadIdx.x == 0) tl[5] = clock64();
+    GACONV_TL(5, threadIdx.x == 0);
     const int rows = min(P.m, g.k - k0), cols = P.rc * nmma;
     const int q_per_row = cols >> 2, quads = rows * q_per_row;
     const int slice = (quads + cl - 1) / cl;
     const int f_begin = min(quads, rank * slice), f_end = min(quads, f_begin + slice);
-    const size_t kcrs = (size_t)g.k * g.r * g.s * g.c;
     const bool direct = groups_per_tile == 1;
-    float* out = direct ? dw : partial + (size_t)cgroup * kcrs;
-    const float scale = direct ? g.alpha : 1.0f;
     const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
-    auto out_offset = [&](int f, int& c, int& valid) -> size_t {     // quad f -> offset of its first element in dW's layout
-        const int row = f / q_per_row, col = (f - row * q_per_row) << 2;
-        const int rl = col / nmma, sc = col - rl * nmma, s_ = sc / P.ct;
-        c = c0 + sc - s_ * P.ct;
-        valid = max(0, min(4, g.c - c));
-        return (size_t)(k0 + row) * g.ws_k + (size_t)(r_lo + rl) * g.ws_r + (size_t)s_ * g.ws_s + (size_t)c * g.ws_c;
+    // quad index -> (row, quad column) without a division per element: a thread's indices advance by the block size
+    const int step_r = (int)blockDim.x / q_per_row, step_q = (int)blockDim.x - step_r * q_per_row;
+    const int f_first = f_begin + (int)threadIdx.x;
+    const int row_first = f_first / q_per_row, cq_first = f_first - row_first * q_per_row;
+    auto store_dw = [&](int row, int cq, const float4& t) {      // alpha * t -> the four elements of (row, quad column cq)
+        int sc = cq << 2, rl = 0;
+        while (sc >= nmma) { sc -= nmma; ++rl; }
+        const int s_ = sc >> P.ct_shift, c = c0 + (sc & (P.ct - 1));
+        const int valid = min(4, g.c - c);
+        const size_t off = (size_t)(k0 + row) * g.ws_k + (size_t)(r_lo + rl) * g.ws_r + (size_t)s_ * g.ws_s + (size_t)c * g.ws_c;
+        const float a = g.alpha;
+        if (vec && valid == 4) {
+            *reinterpret_cast<float4*>(dw + off) = make_float4(a * t.x, a * t.y, a * t.z, a * t.w);
+        } else {
+            const float tv[4] = {t.x, t.y, t.z, t.w};
+            for (int j = 0; j < valid; ++j) dw[off + (size_t)j * g.ws_c] = a * tv[j];
+        }
     };
+    float4* slot = reinterpret_cast<float4*>(partial) + ((size_t)tile * groups_per_tile + cgroup) * P.slot_quads;
     if (!s_abort) {
-        for (int f = f_begin + (int)threadIdx.x; f < f_end; f += blockDim.x) {
-            const int row = f / q_per_row, col = (f - row * q_per_row) << 2;
-            const float* src = red + row * red_stride + col;
+        int row = row_first, cq = cq_first;
+        for (int f = f_first; f < f_end; f += blockDim.x) {
+            const float* src = red + row * red_stride + (cq << 2);
             float4 v[4];                                            // all ranks' pieces first (cl <= 4), then the sum in rank order
 #pragma unroll
             for (int rk = 0; rk < 4; ++rk)
@@ -345,19 +420,42 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             float4 t = v[0];
 #pragma unroll
             for (int rk = 1; rk < 4; ++rk) { t.x += v[rk].x; t.y += v[rk].y; t.z += v[rk].z; t.w += v[rk].w; }
-            int c, valid;
-            const size_t off = out_offset(f, c, valid);
-            if (vec && valid == 4) {
-                *reinterpret_cast<float4*>(out + off) = make_float4(scale * t.x, scale * t.y, scale * t.z, scale * t.w);
-            } else {
-                const float tv[4] = {t.x, t.y, t.z, t.w};
-                for (int j = 0; j < valid; ++j) out[off + (size_t)j * g.ws_c] = scale * tv[j];
+            if (direct) store_dw(row, cq, t);
+            else slot[f] = t;
+            row += step_r; cq += step_q;
+            if (cq >= q_per_row) { cq -= q_per_row; ++row; }
+        }
+    }
+    GACONV_TL(6, threadIdx.x == 0);
+    if (!direct) {
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t* ctr = counters + tile * cl + rank;
+            const uint32_t ticket = atomicAdd(ctr, 1u);
+            s_last = ticket == (uint32_t)groups_per_tile - 1;
+            if (s_last) *ctr = 0;                                   // every cluster has arrived: leave the counter as found
+        }
+        __syncthreads();
+        if (s_last && !s_abort) {
+            __threadfence();
+            const float4* slot0 = reinterpret_cast<const float4*>(partial) + (size_t)tile * groups_per_tile * P.slot_quads;
+            int row = row_first, cq = cq_first;
+            for (int f = f_first; f < f_end; f += blockDim.x) {
+                float4 t = __ldcg(slot0 + f);
+#pragma unroll 4
+                for (int gi = 1; gi < groups_per_tile; ++gi) {
+                    const float4 u = __ldcg(slot0 + (size_t)gi * P.slot_quads + f);
+                    t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+                }
+                store_dw(row, cq, t);
+                row += step_r; cq += step_q;
+                if (cq >= q_per_row) { cq -= q_per_row; ++row; }
             }
         }
     }
-    if (tl && threadIdx.x == 0) tl[6] = clock64();
     if (cl > 1) cluster.sync();      // peers may still be reading this CTA's block
-    if (tl && threadIdx.x == 0) tl[7] = clock64();
+    GACONV_TL(7, threadIdx.x == 0);
 }
 
 // dYt[n][j][k] = dY[n][k][j] for maps of fewer than 16 pixels (the map is too short for a TMA row).
@@ -382,7 +480,25 @@ CUtensorMapSwizzle swizzle_for(int bytes) {
 }
 int swz_code(int bytes) { return bytes == 128 ? 2 : bytes == 64 ? 4 : 6; }
 int pow2_ceil(int v) { int p = 32; while (p < v) p *= 2; return p; }
+#ifdef GACONV_TUNING
 int env_int(const char* name, int dflt) { const char* e = getenv(name); return e ? atoi(e) : dflt; }
+#else
+constexpr int env_int(const char*, int dflt) { return dflt; }
+#endif
+
+// SMs of the current device (one CTA of this kernel fills an SM)
+int sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 }  // namespace
 
@@ -415,16 +531,22 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.rsplit = (g.c >= 64 && g.r > 1 && env_int("GACONV_TC_RSPLIT", 1)) ? 1 : 0;
     P.rc = P.rsplit ? 1 : g.r;
     if (P.rsplit) P.m = g.k <= 64 ? 64 : 128;
+    // One filter row per CTA means one accumulator and one issuing thread, which cannot keep the tensor pipe
+    // busy (an MMA of N <= 256 executes in about the time one thread needs to issue it).  So the CTA keeps
+    // two accumulators for the row and two issuers take alternate chunks.
+    P.dual = (P.rc == 1 && env_int("GACONV_TC_DUAL", 1)) ? 1 : 0;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     P.tiny = tiny ? 1 : 0;
     P.by_image = small_map ? 1 : 0;
     // channels per tile: one swizzle span wide (16, 32 or 64 channels), limited by MMA N <= 256 and TMEM columns
     int ct = g.c >= 64 ? 64 : g.c >= 32 ? 32 : 16;
-    auto cols_for = [&](int c) { return (P.m == 128 ? P.rc : (P.rc + 1) / 2) * g.s * c; };
+    const int accs = P.dual ? 2 : P.rc;                 // accumulators of a CTA
+    auto cols_for = [&](int c) { return (P.m == 128 ? accs : (accs + 1) / 2) * g.s * c; };
     while (ct > 16 && (g.s * ct > 256 || cols_for(ct) > 512)) ct /= 2;
     if (g.s * ct > 256 || cols_for(ct) > 512) return false;
     if ((g.s * ct) % (P.m == 128 ? 16 : 8) != 0) return false;
     P.ct = ct;
+    P.ct_shift = ct == 64 ? 6 : ct == 32 ? 5 : 4;
     P.tiles_k = (g.k + P.m - 1) / P.m;
     P.tiles_c = (g.c + ct - 1) / ct;
     if (P.rsplit) halo = false;          // a single row needs no halo rows: its S tiles are loaded directly
@@ -436,8 +558,9 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.wide = (env_int("GACONV_TC_WIDE", 1) && !small_map && g.stride_h == 1 && (g.q % 16 == 0 || g.q == 8) && 64 % g.q == 0) ? 1 : 0;
     P.b_tiles = P.wide ? 1 : halo ? g.s : P.rc * g.s;
 
-    // chunk size: as many rows (or images) as fit a ~48 KiB stage
-    const int budget = env_int("GACONV_TC_STAGE_KB", 48) * 1024;
+    // chunk size: as many rows (or images) as fit the stage budget.  The hand-over of a stage costs the producer
+    // and the issuer several hundred cycles each, so a stage should carry at least ~8 MMAs.
+    const int budget = env_int("GACONV_TC_STAGE_KB", 64) * 1024;
     auto stage_bytes = [&](int ci, int bp, int* a_subs, int* tile_bytes, int* tile_stride) {
         const int px = ci * bp * g.q;
         *a_subs = tiny ? px / 64 : small_map ? ci : px / 64;
@@ -457,55 +580,67 @@ bool plan_tc(const Geom& g, TcPlan* out)
         while (bp * 2 <= g.p && g.p % (bp * 2) == 0 && (halo ? bp * 2 + g.r - 1 : bp * 2 * g.stride_h) <= 256 &&
                stage_bytes(1, bp * 2, &a_subs, &tb, &ts) <= budget) bp *= 2;
         if (g.p % bp != 0) return false;
+        // whole maps that are still small: several images per chunk (the wide tile of a single filter row has no
+        // halo rows, so the images of a chunk are contiguous in shared memory and the descriptors just keep advancing)
+        if (bp == g.p && P.wide && P.rc == 1)
+            while (ci * 2 <= 8 && ci * 2 <= g.n && stage_bytes(ci * 2, bp, &a_subs, &tb, &ts) <= budget) ci *= 2;
     }
     P.ci = ci; P.bp = bp;
     P.stage_bytes = stage_bytes(ci, bp, &a_subs, &tb, &ts);
     P.stage_bytes = (P.stage_bytes + 1023) / 1024 * 1024;
     P.a_subs = a_subs; P.b_tile_bytes = tb; P.b_tile_stride = ts;
+    P.a_subs_img = (tiny || small_map) ? a_subs : a_subs / ci;
     P.a_sub_bytes = tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
     P.a_k4_step = tiny ? (16 * 128) >> 4 : 2;
     P.a_lbo = tiny ? ci * pq * 128 : 16;               // tiny: bytes between the 64-channel atoms of an A tile
     P.a_region_bytes = ((tiny ? (P.m / 64) * ci * pq * 128 : P.a_subs * P.a_sub_bytes) + 1023) / 1024 * 1024;
     P.ksteps = ci * bp * g.q / 16;
-    P.chunks = small_map ? (g.n + ci - 1) / ci : g.n * (g.p / bp);
+    P.chunks = (small_map || ci > 1) ? (g.n + ci - 1) / ci : g.n * (g.p / bp);
     const int smem_budget = 200 * 1024;
     P.stages = smem_budget / P.stage_bytes;
     if (P.stages > kMaxStages) P.stages = kMaxStages;
     if (P.stages < 2) return false;
-    P.issuers = P.rc < 3 ? P.rc : 3;
+    P.issuers = P.dual ? 2 : P.rc < 3 ? P.rc : 3;
     P.tmem_cols = pow2_ceil(cols_for(ct));
     if (P.tmem_cols > 512) return false;
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
     P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((tiny ? 1u : 0u) << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
-    // Splits of the reduction: about 128 CTAs in all, in clusters of up to 4 consecutive splits that reduce
-    // through distributed shared memory (clusters of 8 full-SM CTAs measured slower: they are placed GPC by GPC).
+    // Splits of the reduction: one CTA per SM in all.  Consecutive splits form a thread-block cluster of up to 4
+    // that reduces through distributed shared memory (clusters of 8 full-SM CTAs measured slower: they are
+    // placed GPC by GPC); the clusters of a tile meet in the workspace.
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
-    int cl = 1;
-    while (cl * 2 <= 8 && tiles * cl * 2 <= 128 && cl * 2 <= P.chunks) cl *= 2;
-    if (cl > 4) cl = 4;      // the reduction loop holds one piece per rank in registers
-    if (env_int("GACONV_TC_CLUSTER", 4) < cl) cl = env_int("GACONV_TC_CLUSTER", 4) < 1 ? 1 : env_int("GACONV_TC_CLUSTER", 4);
-    int splits = env_int("GACONV_TC_SPLITS", 0);
-    if (splits <= 0) {
-        splits = 128 / tiles;
-        if (splits < 1) splits = 1;
+    const int sms = sm_count();
+    int max_splits = env_int("GACONV_TC_SPLITS", 0);
+    if (max_splits <= 0) {
+        max_splits = sms / tiles;
+        if (max_splits < 1) max_splits = 1;
         // the cluster slots are written and read back (mostly in L2): cap them only where they would dwarf the inputs
         const size_t out_bytes = (size_t)g.k * g.r * g.s * g.c * 4;
         const size_t in_bytes = ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 2;
-        while (splits > cl && (size_t)(splits / cl) * out_bytes > 4 * in_bytes + (8u << 20)) --splits;
+        while (max_splits > 4 && (size_t)(max_splits / 4) * out_bytes > 4 * in_bytes + (8u << 20)) --max_splits;
     }
-    if (splits > P.chunks) splits = P.chunks;
-    splits = splits / cl * cl;                       // whole clusters
-    if (splits < cl) splits = cl;
+    if (max_splits > P.chunks) max_splits = P.chunks;
+    // cluster size: the largest of 4, 3, 2, 1 that loses at most a tenth of the CTAs to rounding
+    const int cl_cap = env_int("GACONV_TC_CLUSTER", 4);
+    int cl = 1, splits = max_splits;
+    for (int c = 4; c >= 1; --c) {
+        if (c > cl_cap || c > max_splits) continue;
+        const int sp = max_splits / c * c;
+        if (sp * 10 >= max_splits * 9) { cl = c; splits = sp; break; }
+    }
     P.cl = cl;
     P.splits = splits;
+    P.chunk_base = P.chunks / splits;
+    P.chunk_rem = P.chunks - P.chunk_base * splits;
     // the reduction block must fit the dynamic shared memory (it reuses the operand stages)
     const size_t red_bytes = (size_t)P.m * (P.rc * g.s * ct + 4) * 4;
     if (red_bytes > 212 * 1024) return false;
     if ((size_t)tiles * cl > kWsNumCounters) return false;
+    P.slot_quads = P.m * (P.rc * g.s * ct / 4);
     P.timeline = env_int("GACONV_TC_TIMELINE", 0);
 
-    out->partial_bytes = splits / cl > 1 ? (size_t)(splits / cl) * g.k * g.r * g.s * g.c * 4 : 0;
+    out->partial_bytes = splits / cl > 1 ? (size_t)tiles * (splits / cl) * P.slot_quads * 16 : 0;
     out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
     memcpy(out->opaque, &P, sizeof(P));
@@ -564,14 +699,16 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     smem += 1024 + (size_t)P.m * 128;
     dim3 grid(P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1), P.splits);
     const int ks = P.a_sub_px / 16;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
     cudaError_t err = cudaErrorInvalidValue;
 #define GACONV_TC_CASE(RR, KK)                                                                                     \
     if (err == cudaErrorInvalidValue && (RR == 0 || (P.rc == RR && ks == KK))) {                                     \
-        static size_t configured = 0;                                                                              \
+        static size_t configured[64] = {};           /* the attribute is per device */                            \
         err = cudaSuccess;                                                                                         \
-        if (smem > configured) {                                                                                   \
+        if (dev < 0 || dev >= 64 || smem > configured[dev]) {                                                      \
             err = cudaFuncSetAttribute(exact_tc_kernel<RR, KK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-            if (err == cudaSuccess) configured = smem;                                                             \
+            if (err == cudaSuccess && dev >= 0 && dev < 64) configured[dev] = smem;                                \
         }                                                                                                          \
         if (err == cudaSuccess) {                                                                                  \
             err = launch_kernel(exact_tc_kernel<RR, KK>, grid, dim3(256), smem, stream, dim3(1, P.cl, 1), map_dy, map_x, dw, \
@@ -586,9 +723,6 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
 #undef GACONV_TC_CASE
     if (err != cudaSuccess) return err;
     note_launch();
-    if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
-    if (P.splits / P.cl > 1)
-        return reduce_splits(partial, dw, (size_t)g.k * g.r * g.s * g.c, P.splits / P.cl, g.alpha, stream);
     return cudaGetLastError();
 }
 
