@@ -15,9 +15,12 @@
 //        the 32 lanes of each TMEM sub-partition, so two accumulators share the same columns.
 // A CTA owns one (k-tile, c-tile) block of dW and a contiguous range of reduction chunks.  Consecutive
 // splits form a thread-block cluster and add their blocks through distributed shared memory; if a tile
-// has several clusters, each cluster leaves its sum in a slot of the workspace and the last cluster of
-// the tile to finish a slice adds the slots of that slice in slot order (a ticket per slice), so the
-// order of every sum is fixed whatever the timing.
+// has several clusters, each cluster leaves its sum in a slot of the workspace and a second, small kernel
+// (reduce_slots_kernel, launched as a programmatic dependent so its start-up overlaps) adds the slots with
+// the whole GPU, in an order that depends only on the launch geometry.  No CTA waits for a CTA outside
+// its cluster.  (Summing in the same kernel -- by the last cluster to arrive, or by all CTAs of a tile
+// once a counter shows them complete -- measured slower: the first serialises megabytes of slot reads on
+// a few CTAs, the second needs the whole grid resident, which cluster placement does not guarantee.)
 //
 // Warp roles: warp 0 = TMA producer; warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns
 // the TMEM allocation); warps 4..7 = epilogue.  The filter rows are dealt round-robin to the issuers:
@@ -30,6 +33,8 @@
 
 #include <cooperative_groups.h>
 
+#include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -39,7 +44,9 @@
 // GACONV_TUNING builds carry clock64 stamps of CTA (0,0)'s phases (workspace bytes [64,128)) and read
 // planner overrides from the environment; the default build has neither.
 #ifdef GACONV_TUNING
-#define GACONV_TL(slot, cond) do { if (tl && (cond)) tl[slot] = clock64(); } while (0)
+#define GACONV_TL(slot, cond) do { if (tl && (cond)) tl[slot] = clock64(); if (P.timeline && threadIdx.x == 128) gaconv_tuning_stamps[(blockIdx.y * gridDim.x + blockIdx.x) & 1023][slot] = gaconv_globaltimer(); } while (0)
+__device__ unsigned long long gaconv_tuning_stamps[1024][8];
+__device__ __forceinline__ unsigned long long gaconv_globaltimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #else
 #define GACONV_TL(slot, cond) do { } while (0)
 #endif
@@ -110,11 +117,14 @@ struct TcParams {
     int dual;           // 1 (only with rc == 1): two accumulators, issuer i takes the chunks with (index & 1) == i
     int issuers;        // MMA-issuing warps: min(R, 3), or 2 when dual; issuer i takes filter rows i, i+issuers, ...
     int slot_quads;     // float4 elements of one cluster slot (m rows x rc * s * ct columns)
+    uint32_t qpr_magic; // ceil(2^32 / quads per row): quad index -> row by one multiply
+    int reduce_parts;   // grid.x of reduce_slots_kernel
     uint32_t idesc;
     int timeline;       // tuning builds: CTA (0,0) records clock64 stamps of its phases at workspace bytes [64, 128)
 };
 
 constexpr int kMaxStages = 8;
+constexpr int kMaxQuadCols = 7 * 256 / 4;      // rc <= 7 filter rows of at most 256 columns
 
 // R_T: filter rows (0 = take it from the geometry); KS_T: k-steps per A box (0 = from the plan).
 // The compile-time values let the issue loop unroll into straight-line MMA instructions.
@@ -128,7 +138,10 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ int s_last;
+    // for quad column cq of the CTA's block: offset of its first element within a dW row block, and how many of
+    // its four channels exist (the last channel tile may be partial)
+    __shared__ int s_coloff[kMaxQuadCols];
+    __shared__ signed char s_colvalid[kMaxQuadCols];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -144,7 +157,15 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));   // reduction block, aliases the stages
     const int red_stride = P.rc * nmma + 4;
 
+#ifdef GACONV_TUNING
+    if (P.timeline && threadIdx.x == 128) gaconv_tuning_stamps[(blockIdx.y * gridDim.x + blockIdx.x) & 1023][1] = gaconv_globaltimer();
+#endif
     pdl_release_next_grid();
+    for (int cq = threadIdx.x; cq < (P.rc * nmma) >> 2; cq += blockDim.x) {
+        const int col = cq << 2, rl = col / nmma, sc = col - rl * nmma, s_ = sc >> P.ct_shift, c = c0 + (sc & (P.ct - 1));
+        s_coloff[cq] = (int)((r_lo + rl) * g.ws_r + s_ * g.ws_s + c * g.ws_c);
+        s_colvalid[cq] = (signed char)max(0, min(4, g.c - c));
+    }
     if (threadIdx.x == 0) {
         // the tensor maps are kernel parameters: fetching them does not depend on the previous kernel
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_dy) : "memory");
@@ -168,49 +189,62 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
 #endif
     GACONV_TL(0, threadIdx.x == 0);
 
-    if (warp == 0 && lane == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        // chunk coordinates advance incrementally: no division inside the loop
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (whole warp)
+        // Lane 0 waits for the stage and posts the byte count; then lane b issues copy b of the chunk, so the
+        // copies of a stage leave together instead of one after the other from a single thread.
+        // Chunk coordinates advance incrementally: no division inside the loop for the first 32 copies.
         int n0, p0;
         const bool whole_maps = P.by_image != 0 || P.ci > 1;
         const int cpi = whole_maps ? 1 : g.p / P.bp;
         if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
         const uint32_t tx_bytes = (P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes;
+        const int n_a = P.tiny ? P.m / 64 : P.by_image ? 1 : P.a_subs, n_all = n_a + P.b_tiles;
+        // what copy `lane` is: image and box of an A copy, or filter row and column shift of a B copy
+        const int a_img = (P.tiny || P.by_image) ? 0 : lane / P.a_subs_img, a_sub = (P.tiny || P.by_image) ? 0 : lane - a_img * P.a_subs_img;
+        const int b_idx = lane - n_a, b_rr = b_idx > 0 ? b_idx / g.s : 0, b_ss = b_idx > 0 ? b_idx - b_rr * g.s : 0;
         int issued = 0, st = 0, ph = 0;
         for (int it = 0; it < nchunks; ++it) {
-            if (it >= P.stages && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1)) { s_abort = 1; atomicOr(status, 1u); break; }
-            if (s_abort) break;
             const uint32_t full = smem_u32(&bar_full[st]);
-            const uint32_t sa = smem_base + st * P.stage_bytes;
-            uint32_t sb = sa + P.a_region_bytes;
-            mbar_expect_tx(full, tx_bytes);
-            if (P.tiny) {                                                        // one box per 64-channel atom
-                for (int a = 0; a * 64 < P.m; ++a) tma_load_3d(sa + a * P.a_lbo, &map_dy, full, k0 + 64 * a, 0, n0);
-            } else if (P.by_image) {
-                tma_load_3d(sa, &map_dy, full, 0, k0, n0);                       // ci whole maps in one box
-            } else {
-                uint32_t dst = sa;                                               // images past the batch read as zeros
-                for (int i = 0; i < P.ci; ++i) {
-                    int px = p0 * g.q;
-                    for (int b = 0; b < P.a_subs_img; ++b, px += 64, dst += P.a_sub_bytes) tma_load_3d(dst, &map_dy, full, px, k0, n0 + i);
-                }
+            int ok = 1;
+            if (lane == 0) {
+                if (it >= P.stages && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1)) { s_abort = 1; atomicOr(status, 1u); }
+                if (s_abort) ok = 0;
+                else mbar_expect_tx(full, tx_bytes);
             }
-            if (P.wide) {
-                tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
-            } else if (P.halo) {
-                for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride) tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 - g.pad_h, n0);
-            } else {
-                for (int r = r_lo; r < r_lo + P.rc; ++r)
-                    for (int s = 0; s < g.s; ++s, sb += P.b_tile_stride)
-                        tma_load_4d(sb, &map_x, full, c0, s - g.pad_w, p0 * g.stride_h + r - g.pad_h, n0);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            const uint32_t sa = smem_base + st * P.stage_bytes;
+            const uint32_t sb = sa + P.a_region_bytes;
+            for (int b = lane; b < n_all; b += 32) {
+                if (b < n_a) {
+                    if (P.tiny) {                                                // one box per 64-channel atom
+                        tma_load_3d(sa + b * P.a_lbo, &map_dy, full, k0 + 64 * b, 0, n0);
+                    } else if (P.by_image) {
+                        tma_load_3d(sa, &map_dy, full, 0, k0, n0);               // ci whole maps in one box
+                    } else {                                                     // images past the batch read as zeros
+                        const int i = b < 32 ? a_img : b / P.a_subs_img, sub = b < 32 ? a_sub : b - i * P.a_subs_img;
+                        tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, p0 * g.q + 64 * sub, k0, n0 + i);
+                    }
+                } else {
+                    const int j = b - n_a;
+                    if (P.wide) {
+                        tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
+                    } else if (P.halo) {
+                        tma_load_4d(sb + j * P.b_tile_stride, &map_x, full, c0, j - g.pad_w, p0 - g.pad_h, n0);
+                    } else {
+                        const int rr = b < 32 ? b_rr : j / g.s, ss = b < 32 ? b_ss : j - rr * g.s;
+                        tma_load_4d(sb + j * P.b_tile_stride, &map_x, full, c0, ss - g.pad_w, p0 * g.stride_h + r_lo + rr - g.pad_h, n0);
+                    }
+                }
             }
             ++issued;
             if (whole_maps) n0 += P.ci;
             else { p0 += P.bp; if (p0 >= g.p) { p0 = 0; ++n0; } }
             if (++st == P.stages) { st = 0; ph ^= 1; }
         }
-        if (s_abort) {   // drain: wait (bounded) for the copies already issued
+        if (lane == 0 && s_abort) {   // drain: wait (bounded) for the copies already issued
             for (int it = max(0, issued - P.stages); it < issued; ++it) mbar_wait(smem_u32(&bar_full[it % P.stages]), (it / P.stages) & 1);
         }
     } else if (warp >= 1 && warp <= 3 && warp - 1 < P.issuers && lane == 0) {
@@ -284,33 +318,50 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         }
         umma_commit(smem_u32(&bar_acc));             // accumulators complete
         GACONV_TL(2, issuer == 0);
-    } else if (warp >= 4) {
+    }
+    __syncwarp();
+    const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
+    auto store_dw = [&](int row, int cq, const float4& t) {      // alpha * t -> the four elements of (row, quad column cq)
+        float* p = dw + (size_t)(k0 + row) * g.ws_k + s_coloff[cq];
+        const int valid = s_colvalid[cq];
+        const float a = g.alpha;
+        if (vec && valid == 4) {
+            *reinterpret_cast<float4*>(p) = make_float4(a * t.x, a * t.y, a * t.z, a * t.w);
+        } else {
+            const float tv[4] = {t.x, t.y, t.z, t.w};
+            for (int j = 0; j < valid; ++j) p[(size_t)j * g.ws_c] = a * tv[j];
+        }
+    };
+    {
         // ------------------------------------------------------------------ epilogue 1: TMEM -> shared memory
         // The accumulators go to a [row][column] fp32 block in this CTA's shared memory (the operand
         // stages are free by now); column = local filter row * nmma + s * ct + c.  Rows are padded by four
         // floats so that the 32 lanes of a warp, one row each, store 16-byte pieces without bank conflicts.
+        // All eight warps take part (the producer and the issuers are done): warps w and w + 4 read the same
+        // 32 lanes of tensor memory and take alternate 16-column pieces.
         const bool ready = mbar_wait_sleepy(smem_u32(&bar_acc), 0);
         if (!ready) { s_abort = 1; atomicOr(status, 1u); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         GACONV_TL(3, threadIdx.x == 128);
-        if (ready && !s_abort) {
-            const int sp = warp & 3;
+        if (__all_sync(0xffffffffu, ready && !s_abort)) {       // warp-uniform: the tensor-memory loads are warp-wide
+            const int sp = warp & 3, half = warp < 4 ? 1 : 0;
+            const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
+            const uint32_t tlane = tmem_base + ((uint32_t)(32 * sp) << 16);
+            const int pieces = nmma >> 4;                      // 16-column pieces per accumulator
             if (P.dual) {
                 // accumulator 0 (even chunks) + accumulator 1 (odd chunks).  M = 128: they sit side by side in the
                 // columns; M = 64: in the two 16-lane halves of each sub-partition (lane l and lane l + 16).
                 const bool has0 = nchunks > 0, has1 = nchunks > 1;
-                const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
                 const bool row_ok = k0 + row < g.k && (P.m == 128 || lane < 16);
-                const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16);
                 float* rrow = red + row * red_stride;
-                for (int col = 0; col < nmma; col += 32) {
+                for (int pc = half; pc < pieces; pc += 4) {     // this warp: pieces pc and pc + 2
                     float v0[2][16], v1[2][16];
-                    const int nld = min(2, (nmma - col) >> 4);
+                    const int nld = pc + 2 < pieces ? 2 : 1;
 #pragma unroll
                     for (int u = 0; u < 2; ++u)
                         if (u < nld) {
-                            tmem_ld16_nowait(tbase + col + 16 * u, v0[u]);
-                            if (P.m == 128) tmem_ld16_nowait(tbase + nmma + col + 16 * u, v1[u]);
+                            tmem_ld16_nowait(tlane + 16 * (pc + 2 * u), v0[u]);
+                            if (P.m == 128) tmem_ld16_nowait(tlane + nmma + 16 * (pc + 2 * u), v1[u]);
                         }
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
@@ -324,35 +375,34 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                             t[e] = (has0 ? a0 : 0.f) + (has1 ? a1 : 0.f);
                         }
                         if (!row_ok) continue;
-                        float4* p4 = reinterpret_cast<float4*>(rrow + col + 16 * u);
+                        float4* p4 = reinterpret_cast<float4*>(rrow + 16 * (pc + 2 * u));
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) p4[q4] = make_float4(t[4 * q4], t[4 * q4 + 1], t[4 * q4 + 2], t[4 * q4 + 3]);
                     }
                 }
             } else {
                 const int groups = P.m == 128 ? P.rc : (P.rc + 1) / 2;
-                const int row = P.m == 128 ? 32 * sp + lane : 16 * sp + (lane & 15);
                 for (int gi = 0; gi < groups; ++gi) {
                     const int rl = P.m == 128 ? gi : 2 * gi + (lane >> 4);      // row within this CTA's filter rows
                     const bool row_ok = rl < P.rc && k0 + row < g.k;
-                    const uint32_t tbase = tmem_base + ((uint32_t)(32 * sp) << 16) + gi * nmma;
                     float* rrow = red + row * red_stride + rl * nmma;
-                    for (int col = 0; col < nmma; col += 64) {
+                    for (int pc = half; pc < pieces; pc += 8) {                 // this warp: pieces pc, pc + 2, pc + 4, pc + 6
                         float v[4][16];                                        // up to four 16-column loads in flight
-                        const int nld = min(4, (nmma - col) >> 4);
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
-                            if (u < nld) tmem_ld16_nowait(tbase + col + 16 * u, v[u]);
+                            if (pc + 2 * u < pieces) tmem_ld16_nowait(tlane + gi * nmma + 16 * (pc + 2 * u), v[u]);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                         if (!row_ok) continue;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            if (u >= nld) continue;
-                            float4* p4 = reinterpret_cast<float4*>(rrow + col + 16 * u);
+                            if (pc + 2 * u >= pieces) continue;
+                            float4* p4 = reinterpret_cast<float4*>(rrow + 16 * (pc + 2 * u));
 #pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4)
-                                p4[q4] = nchunks > 0 ? make_float4(v[u][4 * q4], v[u][4 * q4 + 1], v[u][4 * q4 + 2], v[u][4 * q4 + 3])
-                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+                            for (int q4 = 0; q4 < 4; ++q4) {
+                                const float4 t4 = nchunks > 0 ? make_float4(v[u][4 * q4], v[u][4 * q4 + 1], v[u][4 * q4 + 2], v[u][4 * q4 + 3])
+                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                                p4[q4] = t4;
+                            }
                         }
                     }
                 }
@@ -373,10 +423,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     // The cl CTAs of a cluster are consecutive splits of one output tile.  After a cluster barrier CTA
     // `rank` adds slice `rank` of the block over the cl CTAs through distributed shared memory, in
     // rank order.  With one cluster per tile the result (times alpha) goes straight to dW; with several,
-    // to the cluster's slot in the workspace, and the last cluster of the tile to deliver slice `rank`
-    // (a ticket per tile and slice) adds that slice over the slots in slot order and writes dW.
-    // A CTA that gave up on a wait still takes part in the barriers and the ticket, so its peers never
-    // wait in vain and the counters return to zero.
+    // to the cluster's slot in the workspace, which reduce_slots_kernel adds up afterwards.
+    // A CTA that gave up on a wait still takes part in the barriers, so its peers never wait in vain.
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     const int cl = P.cl, rank = cl > 1 ? (int)cluster.block_rank() : 0;
@@ -388,90 +436,132 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int slice = (quads + cl - 1) / cl;
     const int f_begin = min(quads, rank * slice), f_end = min(quads, f_begin + slice);
     const bool direct = groups_per_tile == 1;
-    const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
-    // quad index -> (row, quad column) without a division per element: a thread's indices advance by the block size
-    const int step_r = (int)blockDim.x / q_per_row, step_q = (int)blockDim.x - step_r * q_per_row;
-    const int f_first = f_begin + (int)threadIdx.x;
-    const int row_first = f_first / q_per_row, cq_first = f_first - row_first * q_per_row;
-    auto store_dw = [&](int row, int cq, const float4& t) {      // alpha * t -> the four elements of (row, quad column cq)
-        int sc = cq << 2, rl = 0;
-        while (sc >= nmma) { sc -= nmma; ++rl; }
-        const int s_ = sc >> P.ct_shift, c = c0 + (sc & (P.ct - 1));
-        const int valid = min(4, g.c - c);
-        const size_t off = (size_t)(k0 + row) * g.ws_k + (size_t)(r_lo + rl) * g.ws_r + (size_t)s_ * g.ws_s + (size_t)c * g.ws_c;
-        const float a = g.alpha;
-        if (vec && valid == 4) {
-            *reinterpret_cast<float4*>(dw + off) = make_float4(a * t.x, a * t.y, a * t.z, a * t.w);
-        } else {
-            const float tv[4] = {t.x, t.y, t.z, t.w};
-            for (int j = 0; j < valid; ++j) dw[off + (size_t)j * g.ws_c] = a * tv[j];
-        }
-    };
+    // quad index -> (row, quad column) by a multiply with the rounded-up reciprocal (exact for these ranges), so the
+    // iterations below are independent and the compiler keeps several quads in flight
+    const uint32_t qpr_magic = P.qpr_magic;
+    auto quad_row = [&](int f) { return (int)__umulhi((uint32_t)f, qpr_magic); };
     float4* slot = reinterpret_cast<float4*>(partial) + ((size_t)tile * groups_per_tile + cgroup) * P.slot_quads;
     if (!s_abort) {
-        int row = row_first, cq = cq_first;
-        for (int f = f_first; f < f_end; f += blockDim.x) {
-            const float* src = red + row * red_stride + (cq << 2);
-            float4 v[4];                                            // all ranks' pieces first (cl <= 4), then the sum in rank order
-#pragma unroll
-            for (int rk = 0; rk < 4; ++rk)
-                v[rk] = rk >= cl ? make_float4(0.f, 0.f, 0.f, 0.f)
-                                 : cl > 1 ? ld_dsmem_f4(smem_u32(src), (uint32_t)rk) : *reinterpret_cast<const float4*>(src);
-            float4 t = v[0];
-#pragma unroll
-            for (int rk = 1; rk < 4; ++rk) { t.x += v[rk].x; t.y += v[rk].y; t.z += v[rk].z; t.w += v[rk].w; }
-            if (direct) store_dw(row, cq, t);
-            else slot[f] = t;
-            row += step_r; cq += step_q;
-            if (cq >= q_per_row) { cq -= q_per_row; ++row; }
-        }
-    }
-    GACONV_TL(6, threadIdx.x == 0);
-    if (!direct) {
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t* ctr = counters + tile * cl + rank;
-            const uint32_t ticket = atomicAdd(ctr, 1u);
-            s_last = ticket == (uint32_t)groups_per_tile - 1;
-            if (s_last) *ctr = 0;                                   // every cluster has arrived: leave the counter as found
-        }
-        __syncthreads();
-        if (s_last && !s_abort) {
-            __threadfence();
-            const float4* slot0 = reinterpret_cast<const float4*>(partial) + (size_t)tile * groups_per_tile * P.slot_quads;
-            int row = row_first, cq = cq_first;
-            for (int f = f_first; f < f_end; f += blockDim.x) {
-                float4 t = __ldcg(slot0 + f);
+        const int f_first = f_begin + (int)threadIdx.x;
+        if (cl == 1) {
 #pragma unroll 4
-                for (int gi = 1; gi < groups_per_tile; ++gi) {
-                    const float4 u = __ldcg(slot0 + (size_t)gi * P.slot_quads + f);
-                    t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-                }
-                store_dw(row, cq, t);
-                row += step_r; cq += step_q;
-                if (cq >= q_per_row) { cq -= q_per_row; ++row; }
+            for (int f = f_first; f < f_end; f += blockDim.x) {
+                const int row = quad_row(f), cq = f - row * q_per_row;
+                const float4 t = *reinterpret_cast<const float4*>(red + row * red_stride + (cq << 2));
+                if (direct) store_dw(row, cq, t);
+                else slot[f] = t;
+            }
+        } else {
+#pragma unroll 2
+            for (int f = f_first; f < f_end; f += blockDim.x) {
+                const int row = quad_row(f), cq = f - row * q_per_row;
+                const uint32_t src = smem_u32(red + row * red_stride + (cq << 2));
+                float4 v[4];                                            // all ranks' pieces first (cl <= 4), then the sum in rank order
+#pragma unroll
+                for (int rk = 0; rk < 4; ++rk) v[rk] = rk < cl ? ld_dsmem_f4(src, (uint32_t)rk) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 t = v[0];
+#pragma unroll
+                for (int rk = 1; rk < 4; ++rk) { t.x += v[rk].x; t.y += v[rk].y; t.z += v[rk].z; t.w += v[rk].w; }
+                if (direct) store_dw(row, cq, t);
+                else slot[f] = t;
             }
         }
     }
-    if (cl > 1) cluster.sync();      // peers may still be reading this CTA's block
+    GACONV_TL(6, threadIdx.x == 0);
+    // this CTA no longer reads its peers' blocks: say so now, and wait for the peers' word only before leaving
+    if (cl > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    if (cl > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // peers may still be reading this CTA's block
     GACONV_TL(7, threadIdx.x == 0);
 }
 
-// dYt[n][j][k] = dY[n][k][j] for maps of fewer than 16 pixels (the map is too short for a TMA row).
-__global__ void __launch_bounds__(256)
-transpose_dy_kernel(const __nv_bfloat16* __restrict__ dy, __nv_bfloat16* __restrict__ dyt, int n, int k, int pq)
+// dYt[n][j][k] = dY[n][k][j] for maps of fewer than 64 pixels (their rows are too short for the copy engine).
+// A block takes 64 channels of one image: their maps are one contiguous piece of dY, read in 16-byte units,
+// turned in shared memory, and written as pq rows of up to 128 bytes.
+__global__ void __launch_bounds__(128)
+transpose_dy_kernel(const __nv_bfloat16* __restrict__ dy, __nv_bfloat16* __restrict__ dyt, int k, int pq)
 {
+    __shared__ __align__(16) unsigned short tile[64 * 32];
     pdl_release_next_grid();
+    const int kgroups = (k + 63) / 64;
+    const int n = blockIdx.x / kgroups, k0 = (blockIdx.x - n * kgroups) * 64, kg = min(64, k - k0);
     pdl_wait_prior_grid();
-    const size_t total = (size_t)n * k * pq;
-    const size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // output index: ((n*pq + j)*k + kk)
-    if (o >= total) return;
-    const int kk = (int)(o % k);
-    const size_t rest = o / k;
-    const int j = (int)(rest % pq);
-    const size_t nn = rest / pq;
-    dyt[o] = dy[(nn * k + kk) * pq + j];
+    const size_t base = ((size_t)n * k + k0) * pq;                 // first element of map (n, k0); a multiple of 8 elements
+    const int elems = kg * pq;
+    for (int v = threadIdx.x; v * 8 < elems; v += blockDim.x)
+        reinterpret_cast<uint4*>(tile)[v] = __ldg(reinterpret_cast<const uint4*>(dy + base) + v);
+    __syncthreads();
+    // item = (pixel j, group of eight channels): eight values at stride pq in the tile -> 16 contiguous bytes of dYt
+    const int k8 = kg >> 3;
+    for (int item = threadIdx.x; item < pq * k8; item += blockDim.x) {
+        const int j = item / k8, q = item - j * k8;
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            w[i] = (uint32_t)tile[(8 * q + 2 * i) * pq + j] | ((uint32_t)tile[(8 * q + 2 * i + 1) * pq + j] << 16);
+        *reinterpret_cast<uint4*>(dyt + ((size_t)n * pq + j) * k + k0 + 8 * q) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// Sum of the cluster slots of every tile, for launches whose tiles have many slots: grid (parts, tiles); a CTA
+// adds part `blockIdx.x` of tile `blockIdx.y` over the slots -- L lanes per quad, lane l taking slots l, l + L, ...
+// in ascending order, eight loads in flight, and a fixed shuffle tree over the lanes -- and writes alpha * sum to dW.
+__global__ void __launch_bounds__(256)
+reduce_slots_kernel(const float4* __restrict__ partial, float* __restrict__ dw, const TcParams P)
+{
+    __shared__ int s_coloff[kMaxQuadCols];
+    __shared__ signed char s_colvalid[kMaxQuadCols];
+    const Geom& g = P.g;
+    const int tile = blockIdx.y;
+    const int r_lo = P.rsplit ? tile % g.r : 0, kc_tile = P.rsplit ? tile / g.r : tile;
+    const int k0 = (kc_tile / P.tiles_c) * P.m, c0 = (kc_tile % P.tiles_c) * P.ct;
+    const int nmma = g.s * P.ct, q_per_row = (P.rc * nmma) >> 2;
+    pdl_release_next_grid();
+    for (int cq = threadIdx.x; cq < q_per_row; cq += blockDim.x) {
+        const int col = cq << 2, rl = col / nmma, sc = col - rl * nmma, s_ = sc >> P.ct_shift, c = c0 + (sc & (P.ct - 1));
+        s_coloff[cq] = (int)((r_lo + rl) * g.ws_r + s_ * g.ws_s + c * g.ws_c);
+        s_colvalid[cq] = (signed char)max(0, min(4, g.c - c));
+    }
+    __syncthreads();
+    pdl_wait_prior_grid();
+    const int groups = P.splits / P.cl;
+    const int quads = min(P.m, g.k - k0) * q_per_row;
+    const int part = (quads + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int p_begin = min(quads, (int)blockIdx.x * part), npart = min(quads, p_begin + part) - p_begin;
+    int lg = 0;
+    while (lg < 5 && (2 << lg) * npart <= (int)blockDim.x && (2 << lg) <= groups) ++lg;
+    const int L = 1 << lg, sl = threadIdx.x & (L - 1), per_pass = (int)blockDim.x >> lg;
+    const float4* slot0 = partial + (size_t)tile * groups * P.slot_quads;
+    const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
+    for (int base = 0; base < npart; base += per_pass) {
+        const int q = base + ((int)threadIdx.x >> lg);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (q < npart) {
+            const float4* src = slot0 + p_begin + q;
+            for (int gi = sl; gi < groups; gi += 8 * L) {
+                float4 u[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) u[j] = gi + j * L < groups ? __ldcg(src + (size_t)(gi + j * L) * P.slot_quads) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { acc.x += u[j].x; acc.y += u[j].y; acc.z += u[j].z; acc.w += u[j].w; }
+            }
+        }
+        for (int off = 1; off < L; off <<= 1) {
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+        }
+        if (sl == 0 && q < npart) {
+            const int f = p_begin + q, row = (int)__umulhi((uint32_t)f, P.qpr_magic), cq = f - row * q_per_row;
+            float* p = dw + (size_t)(k0 + row) * g.ws_k + s_coloff[cq];
+            const int valid = s_colvalid[cq];
+            const float a = g.alpha;
+            if (vec && valid == 4) {
+                *reinterpret_cast<float4*>(p) = make_float4(a * acc.x, a * acc.y, a * acc.z, a * acc.w);
+            } else {
+                const float tv[4] = {acc.x, acc.y, acc.z, acc.w};
+                for (int j = 0; j < valid; ++j) p[(size_t)j * g.ws_c] = a * tv[j];
+            }
+        }
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -498,6 +588,31 @@ int sm_count()
         cached[dev] = n;
     }
     return cached[dev];
+}
+
+// How many clusters of `cl` CTAs of this kernel (one CTA per SM) the current device holds at once.
+int resident_clusters(int cl)
+{
+    static int cached[64][5] = {};
+    if (cl <= 1) return sm_count();
+    int dev = 0;
+    if (cl > 4 || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return sm_count() / cl * 8 / 10;
+    if (cached[dev][cl] == 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1, cl * 64, 1); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 200 * 1024;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = cl; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(exact_tc_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, exact_tc_kernel<0, 0>, &cfg) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            n = sm_count() / cl * 8 / 10;          // no answer: a cautious guess
+        }
+        cached[dev][cl] = n;
+    }
+    return cached[dev][cl];
 }
 
 }  // namespace
@@ -606,39 +721,51 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
     P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((tiny ? 1u : 0u) << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
-    // Splits of the reduction: one CTA per SM in all.  Consecutive splits form a thread-block cluster of up to 4
-    // that reduces through distributed shared memory (clusters of 8 full-SM CTAs measured slower: they are
-    // placed GPC by GPC); the clusters of a tile meet in the workspace.
+    // Splits of the reduction: one wave of CTAs, one per SM.  Consecutive splits form a thread-block cluster of up
+    // to 4 that reduces through distributed shared memory; the clusters of a tile meet in the workspace, where the
+    // second kernel adds them up.  Larger clusters mean less workspace traffic, but fewer resident CTAs (clusters
+    // are placed GPC by GPC: 148 CTAs fit as pairs, 135 as triples, 132 as quadruples).
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
-    const int sms = sm_count();
     int max_splits = env_int("GACONV_TC_SPLITS", 0);
     if (max_splits <= 0) {
-        max_splits = sms / tiles;
+        max_splits = sm_count() / tiles;
         if (max_splits < 1) max_splits = 1;
-        // the cluster slots are written and read back (mostly in L2): cap them only where they would dwarf the inputs
-        const size_t out_bytes = (size_t)g.k * g.r * g.s * g.c * 4;
-        const size_t in_bytes = ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 2;
-        while (max_splits > 4 && (size_t)(max_splits / 4) * out_bytes > 4 * in_bytes + (8u << 20)) --max_splits;
     }
     if (max_splits > P.chunks) max_splits = P.chunks;
-    // cluster size: the largest of 4, 3, 2, 1 that loses at most a tenth of the CTAs to rounding
     const int cl_cap = env_int("GACONV_TC_CLUSTER", 4);
-    int cl = 1, splits = max_splits;
-    for (int c = 4; c >= 1; --c) {
-        if (c > cl_cap || c > max_splits) continue;
-        const int sp = max_splits / c * c;
-        if (sp * 10 >= max_splits * 9) { cl = c; splits = sp; break; }
+    // Measured on the layer shapes of the three networks: a cluster whose splits cover the whole tile (no workspace,
+    // no second kernel) wins even at two thirds of the CTAs; otherwise the largest cluster that keeps 85% of them.
+    const int cl_force = env_int("GACONV_TC_FORCE_CL", 0);
+    int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0}, most = 0;
+    for (int c = 1; c <= 4; ++c) {
+        if (c > cl_cap || c > max_splits || (cl_force && c != cl_force)) continue;
+        per_of[c] = std::min(max_splits / c, resident_clusters(c) / tiles);               // clusters per tile
+        sp_of[c] = per_of[c] * c;
+        most = std::max(most, sp_of[c]);
     }
+    int cl = 0, splits = 0;
+    for (int c = 4; c >= 1 && cl == 0; --c)
+        if (per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
+    for (int c = 4; c >= 1 && cl == 0; --c)
+        if (sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
+    const double best = cl == 0 ? 1e30 : 0.0;
+    if (best == 1e30) return false;
     P.cl = cl;
     P.splits = splits;
+    P.reduce_parts = std::max(1, 2 * sm_count() / tiles);
     P.chunk_base = P.chunks / splits;
     P.chunk_rem = P.chunks - P.chunk_base * splits;
     // the reduction block must fit the dynamic shared memory (it reuses the operand stages)
     const size_t red_bytes = (size_t)P.m * (P.rc * g.s * ct + 4) * 4;
     if (red_bytes > 212 * 1024) return false;
-    if ((size_t)tiles * cl > kWsNumCounters) return false;
-    P.slot_quads = P.m * (P.rc * g.s * ct / 4);
+        P.slot_quads = P.m * (P.rc * g.s * ct / 4);
+    P.qpr_magic = (uint32_t)(((1ull << 32) + (P.rc * g.s * ct / 4) - 1) / (P.rc * g.s * ct / 4));
     P.timeline = env_int("GACONV_TC_TIMELINE", 0);
+#ifdef GACONV_TUNING
+    if (env_int("GACONV_TC_VERBOSE", 0))
+        fprintf(stderr, "plan_tc c%d k%d pq%d: m%d ct%d rsplit%d dual%d wide%d tiny%d ci%d bp%d ksteps%d stage %d B x%d, tiles %d splits %d cl %d chunks %d\n",
+                g.c, g.k, pq, P.m, ct, P.rsplit, P.dual, P.wide, P.tiny, ci, bp, P.ksteps, P.stage_bytes, P.stages, tiles, splits, cl, P.chunks);
+#endif
 
     out->partial_bytes = splits / cl > 1 ? (size_t)tiles * (splits / cl) * P.slot_quads * 16 : 0;
     out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
@@ -659,9 +786,8 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
 
     CUtensorMap map_dy, map_x;
     if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) with 64-channel boxes
-        const size_t total = (size_t)g.n * g.k * pq;
-        if (launch_kernel(transpose_dy_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, stream, dim3(1, 1, 1),
-                          static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.n, g.k, pq) != cudaSuccess)
+        if (launch_kernel(transpose_dy_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
+                          static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.k, pq) != cudaSuccess)
             return cudaErrorLaunchFailure;
         note_launch();
         cuuint64_t dims[3] = {(cuuint64_t)g.k, (cuuint64_t)pq, (cuuint64_t)g.n};
@@ -723,7 +849,21 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
 #undef GACONV_TC_CASE
     if (err != cudaSuccess) return err;
     note_launch();
+    if (P.splits / P.cl > 1) {
+        err = launch_kernel(reduce_slots_kernel, dim3(P.reduce_parts, grid.x), dim3(256), 0, stream, dim3(1, 1, 1),
+                            reinterpret_cast<const float4*>(partial), dw, P);
+        if (err != cudaSuccess) return err;
+        note_launch();
+    }
     return cudaGetLastError();
 }
 
 }  // namespace gaconv
+
+#ifdef GACONV_TUNING
+// tuning builds: global-timer stamps (ns) of every CTA of the last tensor-core launch, [1024][8]
+extern "C" int gaconv_tuning_read_stamps(unsigned long long* host)
+{
+    return (int)cudaMemcpyFromSymbol(host, gaconv_tuning_stamps, sizeof(gaconv_tuning_stamps));
+}
+#endif
