@@ -27,10 +27,14 @@
  * dY" and "full selection == exact", spatially constant X (where Algorithm 1 is
  * exact), published known-answer vectors of the Philox-4x32-10 generator, and
  * the paper's stated counts of approximated layers for its first schedule.
+ * Top-k beyond k = 1 follows a reading the paper does not fix (each retained entry
+ * gets sum/k): pinned only by k = 1 == Algorithm 1, by the sparse-list identity and
+ * by the constant-X case -- "parity unpinned" for the choice of scale itself.
  */
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 typedef struct {
@@ -59,7 +63,7 @@ static double xz(const double *x, const oracle_shape_t *g, int n, int c, int hh,
 
 /* ---------------------------------------------------------------------------
  * Exact filter gradient (the operation in the red box of the paper's Figure 1;
- * Section 2.4: "to compute df we have to convolve I with dO"):
+ * Section 2.4, which states the filter gradient as the convolution of the input with the output gradient):
  *
  *   dw[k,c,r,s] = alpha * sum_{n,p,q} xz[n,c,p*st_h+r-pad_h,q*st_w+s-pad_w] * dy[n,k,p,q]
  *
@@ -101,13 +105,26 @@ int oracle_dw_exact(const double *x, const double *dy, double *dw, double *dnorm
 }
 
 /* ---------------------------------------------------------------------------
- * Selection step of Algorithm 1 (its "arg max abs" and "sum" lines) for every
- * (n, k) pair:
- *   idx[n,k]    = first position j = p*Q+q (row-major scan) of the largest |dy[n,k,:,:]|
+ * Order of magnitudes used by every selection below: the bit pattern of |v| read as
+ * an unsigned integer.  For finite values this is the order of |v| itself; it also
+ * gives -0 = +0, infinity above every finite value and NaNs above infinity (ordered
+ * by payload), so the selected position is defined for any input.  Widening a bf16
+ * or fp32 value to double keeps this order, so the key of the double equals the
+ * order of the keys in the input type.
+ * ------------------------------------------------------------------------- */
+static uint64_t mag_key(double v)
+{
+    uint64_t b;
+    memcpy(&b, &v, sizeof b);
+    return b & 0x7fffffffffffffffull;
+}
+
+/* ---------------------------------------------------------------------------
+ * Selection step of Algorithm 1 for every (n, k) pair:
+ *   idx[n,k]    = position j = p*Q+q of the largest-magnitude element of dy[n,k,:,:];
+ *                 among equal magnitudes the lowest j
  *   sum[n,k]    = signed sum of dy[n,k,:,:]
  *   abssum[n,k] = sum of |dy[n,k,:,:]|   (normaliser only; may be NULL)
- * Tie rule: a later element replaces the current one only when strictly larger
- * in magnitude, so the lowest linear index among equal magnitudes wins.
  * ------------------------------------------------------------------------- */
 void oracle_top1_select(const double *dy, int n_, int k_, int pq, int32_t *idx, double *sum, double *abssum)
 {
@@ -115,13 +132,12 @@ void oracle_top1_select(const double *dy, int n_, int k_, int pq, int32_t *idx, 
         for (int k = 0; k < k_; ++k) {
             const double *m = dy + ((size_t)n * k_ + k) * pq;
             int best = 0;
-            double bestmag = fabs(m[0]);
+            uint64_t bestkey = mag_key(m[0]);
             double t = 0.0, ta = 0.0;
             for (int j = 0; j < pq; ++j) {
-                double a = fabs(m[j]);
-                if (a > bestmag) { bestmag = a; best = j; }
+                if (mag_key(m[j]) > bestkey) { bestkey = mag_key(m[j]); best = j; }
                 t += m[j];
-                ta += a;
+                ta += fabs(m[j]);
             }
             idx[(size_t)n * k_ + k] = best;
             sum[(size_t)n * k_ + k] = t;
@@ -130,14 +146,13 @@ void oracle_top1_select(const double *dy, int n_, int k_, int pq, int32_t *idx, 
 }
 
 /* ---------------------------------------------------------------------------
- * Algorithm 1, "Max Gradient Approximation", step by step in the paper's order:
- *   df = 0
- *   for each output channel k, for each batch element n:
- *       (row, col) = arg max |dO[n,k,:,:]|
- *       sum        = sum of dO[n,k,:,:]
- *       df[k,:,:,:] += I[n,:, patch at (row,col)] * sum
- * The patch is read from the zero-padded input at the same offsets the exact
- * formula uses for output position (row, col): element (r,s) of the patch is
+ * Max-gradient approximation (Section 2.3, Algorithm 1).  What it computes: the
+ * exact filter gradient of a tensor that keeps, for every image n and output channel
+ * k, a single entry of dy[n,k,:,:] -- at the position of the largest magnitude -- and
+ * gives that entry the signed sum of the whole map.  Hence, per (k, n): find the
+ * position, take the sum, and add sum * (the input patch that the exact formula
+ * pairs with that output position) to the gradient of filter k.
+ * The patch comes from the zero-padded input: element (r,s) of it is
  * xz[n, c, row*st_h + r - pad_h, col*st_w + s - pad_w].
  * alpha scales the result (the paper scales by 1/128 = 1/batch, Section 2.3).
  * dnorm (may be NULL) receives |alpha| * sum_n abssum[n,k] * |patch element|.
@@ -153,16 +168,12 @@ int oracle_dw_top1(const double *x, const double *dy, double *dw, double *dnorm,
     for (int k = 0; k < g->k; ++k)
         for (int n = 0; n < g->n; ++n) {
             const double *m = dy + ((size_t)n * g->k + k) * pq;
-            /* arg max abs, first maximum */
             int best = 0;
-            double bestmag = fabs(m[0]);
             for (int j = 1; j < pq; ++j)
-                if (fabs(m[j]) > bestmag) { bestmag = fabs(m[j]); best = j; }
-            /* scalar sum of the channel map */
+                if (mag_key(m[j]) > mag_key(m[best])) best = j;
             double sum = 0.0, asum = 0.0;
             for (int j = 0; j < pq; ++j) { sum += m[j]; asum += fabs(m[j]); }
             int row = best / g->q, col = best % g->q;
-            /* patch accumulate */
             for (int c = 0; c < g->c; ++c)
                 for (int r = 0; r < g->r; ++r)
                     for (int s = 0; s < g->s; ++s) {
@@ -176,9 +187,73 @@ int oracle_dw_top1(const double *x, const double *dy, double *dw, double *dnorm,
 }
 
 /* ---------------------------------------------------------------------------
+ * Top-k variant (Section 2.3 says the method extends to the k largest magnitudes
+ * with an adjusted scale; the scale is not given).  Reading taken here: the `topk`
+ * largest-magnitude entries of a map are retained (equal magnitudes: lower position
+ * first) and each receives sum/topk, so that the retained entries still add up to the
+ * signed sum of the map.  topk = 1 is Algorithm 1.
+ *   idx[(n*K+k)*topk + t] = position of the t-th retained entry, in order of selection.
+ * ------------------------------------------------------------------------- */
+void oracle_topk_select(const double *dy, int n_, int k_, int pq, int topk, int32_t *idx, double *sum, double *abssum)
+{
+    if (topk > pq) topk = pq;
+    for (size_t mi = 0; mi < (size_t)n_ * k_; ++mi) {
+        const double *m = dy + mi * pq;
+        double t = 0.0, ta = 0.0;
+        for (int j = 0; j < pq; ++j) { t += m[j]; ta += fabs(m[j]); }
+        sum[mi] = t;
+        if (abssum) abssum[mi] = ta;
+        for (int sel = 0; sel < topk; ++sel) {
+            int best = -1;
+            for (int j = 0; j < pq; ++j) {
+                int taken = 0;
+                for (int u = 0; u < sel; ++u) if (idx[mi * topk + u] == j) taken = 1;
+                if (taken) continue;
+                if (best < 0 || mag_key(m[j]) > mag_key(m[best])) best = j;
+            }
+            idx[mi * topk + sel] = best;
+        }
+    }
+}
+
+int oracle_dw_topk(const double *x, const double *dy, double *dw, double *dnorm,
+                   const oracle_shape_t *g, double alpha, int topk)
+{
+    if (!shape_ok(g) || topk < 1) return 1;
+    size_t total = (size_t)g->k * g->c * g->r * g->s;
+    memset(dw, 0, total * sizeof(double));
+    if (dnorm) memset(dnorm, 0, total * sizeof(double));
+    int pq = g->p * g->q;
+    if (topk > pq) topk = pq;
+    size_t maps = (size_t)g->n * g->k;
+    int32_t *idx = (int32_t *)malloc(maps * topk * sizeof(int32_t));
+    double *sum = (double *)malloc(maps * sizeof(double)), *asum = (double *)malloc(maps * sizeof(double));
+    if (!idx || !sum || !asum) { free(idx); free(sum); free(asum); return 3; }
+    oracle_topk_select(dy, g->n, g->k, pq, topk, idx, sum, asum);
+    for (int k = 0; k < g->k; ++k)
+        for (int n = 0; n < g->n; ++n) {
+            size_t mi = (size_t)n * g->k + k;
+            double share = sum[mi] / topk, ashare = asum[mi] / topk;
+            for (int t = 0; t < topk; ++t) {
+                int row = idx[mi * topk + t] / g->q, col = idx[mi * topk + t] % g->q;
+                for (int c = 0; c < g->c; ++c)
+                    for (int r = 0; r < g->r; ++r)
+                        for (int s = 0; s < g->s; ++s) {
+                            double v = xz(x, g, n, c, row * g->stride_h + r - g->pad_h, col * g->stride_w + s - g->pad_w);
+                            size_t o = (((size_t)k * g->c + c) * g->r + r) * g->s + s;
+                            dw[o] += alpha * (v * share);
+                            if (dnorm) dnorm[o] += fabs(alpha) * fabs(v) * ashare;
+                        }
+            }
+        }
+    free(idx); free(sum); free(asum);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------
  * Sparse accumulate: the filter gradient of an arbitrary list of retained
  * output-gradient entries (n, k, p, q, value).  Section 2.3: the filter gradient
- * is "calculated from this sparse version of the output gradient tensor".
+ * is the one computed from the sparse version of the output-gradient tensor.
  * With the top-1 list it must equal oracle_dw_top1; with every entry of dy listed
  * it must equal oracle_dw_exact.
  * ------------------------------------------------------------------------- */
@@ -202,7 +277,7 @@ int oracle_dw_sparse(const double *x, const int32_t *en, const int32_t *ek, cons
     return 0;
 }
 
-/* Dense "sparse version of the output gradient" (Section 2.3): sum at idx, 0 elsewhere. */
+/* The sparse version of the output gradient, stored densely (Section 2.3): sum at idx, 0 elsewhere. */
 void oracle_sparsify(const int32_t *idx, const double *sum, int n_, int k_, int pq, double *dy_sparse)
 {
     memset(dy_sparse, 0, (size_t)n_ * k_ * pq * sizeof(double));

@@ -80,6 +80,7 @@ def lib():
         _lib.oracle_dw_exact.restype = ctypes.c_int
         _lib.oracle_dw_top1.restype = ctypes.c_int
         _lib.oracle_dw_sparse.restype = ctypes.c_int
+        _lib.oracle_dw_topk.restype = ctypes.c_int
     return _lib
 
 
@@ -128,6 +129,26 @@ def dw_top1(x, dy, g: Shape, alpha: float = 1.0):
     rc = lib().oracle_dw_top1(_d(x), _d(dy), _d(dw), _d(dn), ctypes.byref(g.c_struct()), ctypes.c_double(alpha))
     if rc:
         raise ValueError("oracle_dw_top1 rejected the shape")
+    return dw, dn
+
+
+def topk_select(dy, topk: int):
+    """Selection of the top-k variant: returns (idx int32 [N,K,topk] in order of selection, sum [N,K], abssum [N,K])."""
+    dy = np.ascontiguousarray(dy, dtype=np.float64)
+    n, k, p, q = dy.shape
+    t = min(topk, p * q)
+    idx = np.empty((n, k, t), dtype=np.int32); s = np.empty((n, k)); a = np.empty((n, k))
+    lib().oracle_topk_select(_d(dy), n, k, p * q, t, idx.ctypes.data_as(_ip), _d(s), _d(a))
+    return idx, s, a
+
+
+def dw_topk(x, dy, g: Shape, topk: int, alpha: float = 1.0):
+    """Top-k variant of Algorithm 1 (each retained entry gets sum/topk): returns (dw, dnorm)."""
+    x = _f64(x, (g.n, g.c, g.h, g.w)); dy = _f64(dy, (g.n, g.k, g.p, g.q))
+    dw = np.empty((g.k, g.c, g.r, g.s)); dn = np.empty_like(dw)
+    rc = lib().oracle_dw_topk(_d(x), _d(dy), _d(dw), _d(dn), ctypes.byref(g.c_struct()), ctypes.c_double(alpha), int(topk))
+    if rc:
+        raise ValueError("oracle_dw_topk rejected its arguments (code %d)" % rc)
     return dw, dn
 
 

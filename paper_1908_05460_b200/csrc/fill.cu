@@ -49,44 +49,72 @@ __device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float& z0, 
     z0 = rho * cs; z1 = rho * sn;
 }
 
-__global__ void __launch_bounds__(256)
-random_kernel(float* __restrict__ dw, size_t count, Geom g, uint32_t key0, uint32_t key1, float std, bool contiguous)
+// philox words of counter j -> four standard normals
+__device__ __forceinline__ void normals4(uint32_t j, uint32_t key0, uint32_t key1, float (&z)[4])
 {
-    pdl_release_next_grid();
-    const size_t j = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (4 * j >= count) return;
-    uint32_t c[4] = {(uint32_t)j, 0u, 0u, 0u};
+    uint32_t c[4] = {j, 0u, 0u, 0u};
     uint32_t k0 = key0, k1 = key1;
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
         philox_round(c, k0, k1);
         k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
     }
-    float z[4];
     box_muller(c[0], c[1], z[0], z[1]);
     box_muller(c[2], c[3], z[2], z[3]);
+}
+
+// dW stored in the logical [k][c][r][s] order: thread j writes elements 4j..4j+3 as one 16-byte store.
+__global__ void __launch_bounds__(256)
+random_kcrs_kernel(float* __restrict__ dw, size_t count, uint32_t key0, uint32_t key1, float std)
+{
+    pdl_release_next_grid();
+    const size_t j = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (4 * j >= count) return;
+    float z[4];
+    normals4((uint32_t)j, key0, key1, z);
     pdl_wait_prior_grid();      // the values need no memory; only the stores wait for the previous kernel
-    if (contiguous && 4 * j + 3 < count) {
+    if (4 * j + 3 < count) {
         reinterpret_cast<float4*>(dw)[j] = make_float4(std * z[0], std * z[1], std * z[2], std * z[3]);
-        return;
-    }
-    // logical [k][c][r][s] position of element 4j, decoded once (32-bit arithmetic when it fits), then
-    // stepped; each element goes to its offset in the chosen dW layout
-    int s, r, cc, k;
-    if (count < (1ull << 31)) {
-        uint32_t rest = (uint32_t)(4 * j);
-        s = rest % (uint32_t)g.s; rest /= (uint32_t)g.s;
-        r = rest % (uint32_t)g.r; rest /= (uint32_t)g.r;
-        cc = rest % (uint32_t)g.c; k = rest / (uint32_t)g.c;
     } else {
-        size_t rest = 4 * j;
-        s = (int)(rest % g.s); rest /= g.s;
-        r = (int)(rest % g.r); rest /= g.r;
-        cc = (int)(rest % g.c); k = (int)(rest / g.c);
+        for (int t = 0; 4 * j + t < count; ++t) dw[4 * j + t] = std * z[t];
     }
-    for (int t = 0; t < 4 && 4 * j + t < count; ++t) {
-        dw[k * g.ws_k + cc * g.ws_c + r * g.ws_r + s * g.ws_s] = std * z[t];
-        if (++s == g.s) { s = 0; if (++r == g.r) { r = 0; if (++cc == g.c) { cc = 0; ++k; } } }
+}
+
+// Any other dW layout.  grid (channel chunks, K): a CTA draws the values of one output channel k and `cc`
+// input channels -- a contiguous range of the logical order, so one Philox call still yields four values --
+// into shared memory as [c][r*s], then writes them in storage order: for every (r,s) the chunk's channels,
+// which in the [k][r][s][c] layout are contiguous (16-byte stores when the chunk allows).
+__global__ void __launch_bounds__(256)
+random_strided_kernel(float* __restrict__ dw, Geom g, int cc, uint32_t key0, uint32_t key1, float std)
+{
+    extern __shared__ float vals[];          // [cc][rs]
+    pdl_release_next_grid();
+    const int rs = g.r * g.s, k = blockIdx.y, c0 = blockIdx.x * cc, cn = min(cc, g.c - c0), len = cn * rs;
+    const size_t first = ((size_t)k * g.c + c0) * rs;       // logical index of the chunk's first element
+    const size_t j0 = first / 4;
+    const int head = (int)(first - 4 * j0);                  // elements of counter j0 that belong to the previous chunk
+    for (int i = threadIdx.x; 4 * i < len + head; i += blockDim.x) {
+        float z[4];
+        normals4((uint32_t)(j0 + i), key0, key1, z);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int e = 4 * i + t - head;
+            if (e >= 0 && e < len) vals[e] = std * z[t];
+        }
+    }
+    __syncthreads();
+    pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const bool vec = g.ws_c == 1 && (cn & 3) == 0 && (c0 & 3) == 0 && ((g.ws_k | g.ws_r | g.ws_s) & 3) == 0;
+    for (int p = warp; p < rs; p += warps) {
+        const int r = p / g.s, s = p - r * g.s;
+        float* row = dw + (size_t)k * g.ws_k + (size_t)r * g.ws_r + (size_t)s * g.ws_s + (size_t)c0 * g.ws_c;
+        if (vec) {
+            for (int c = 4 * lane; c < cn; c += 128)
+                *reinterpret_cast<float4*>(row + c) = make_float4(vals[c * rs + p], vals[(c + 1) * rs + p], vals[(c + 2) * rs + p], vals[(c + 3) * rs + p]);
+        } else {
+            for (int c = lane; c < cn; c += 32) row[(size_t)c * g.ws_c] = vals[c * rs + p];
+        }
     }
 }
 
@@ -104,11 +132,23 @@ cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream)
 cudaError_t launch_random(float* dw, const Geom& g, uint64_t seed, float std, cudaStream_t stream)
 {
     const size_t count = (size_t)g.k * g.c * g.r * g.s;
-    const size_t threads = (count + 3) / 4;
-    const bool contiguous = (g.ws_s == 1 && g.ws_r == g.s && g.ws_c == (long long)g.r * g.s);
+    const bool contiguous = (g.ws_s == 1 && g.ws_r == g.s && g.ws_c == (long long)g.r * g.s && g.ws_k == (long long)g.c * g.r * g.s);
+    const uint32_t key0 = (uint32_t)seed, key1 = (uint32_t)(seed >> 32);
     note_launch();
-    return launch_kernel(random_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, stream, dim3(1, 1, 1), dw, count, g,
-                         (uint32_t)seed, (uint32_t)(seed >> 32), std, contiguous);
+    if (contiguous) {
+        const size_t threads = (count + 3) / 4;
+        return launch_kernel(random_kcrs_kernel, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, stream, dim3(1, 1, 1), dw, count,
+                             key0, key1, std);
+    }
+    // channels per CTA: at most 32 KiB of values, and enough CTAs for the machine when K is small
+    const int rs = g.r * g.s;
+    int cc = g.c;
+    while (cc > 4 && ((size_t)cc * rs * 4 > 32 * 1024 || (long long)g.k * ((g.c + cc - 1) / cc) < 296)) cc = (cc + 1) / 2;
+    cc = (cc + 3) / 4 * 4;
+    if ((size_t)cc * rs * 4 > 48 * 1024) cc = 4;
+    if ((size_t)cc * rs * 4 > 48 * 1024) return cudaErrorInvalidValue;      // filters of thousands of taps: not a case this library meets
+    return launch_kernel(random_strided_kernel, dim3((unsigned)((g.c + cc - 1) / cc), (unsigned)g.k), dim3(256), (size_t)cc * rs * 4, stream,
+                         dim3(1, 1, 1), dw, g, cc, key0, key1, std);
 }
 
 }  // namespace gaconv

@@ -132,3 +132,68 @@ def test_metamorphic_relations(g):
 def test_zero_method():
     z = oracle.dw_zero(17)
     assert z.shape == (17,) and np.all(z == 0.0) and not np.any(np.signbit(z))
+
+
+# ---- the order of magnitudes used by the selection: bit pattern of |v| (any input has a defined position) ----
+def test_selection_orders_nan_above_inf_above_finite_and_ignores_the_sign_of_zero():
+    dy = np.zeros((1, 6, 2, 3))
+    dy[0, 0] = [[1.0, -np.inf, 3.0], [np.inf, 2.0, 0.0]]          # two infinities: the earlier one
+    dy[0, 1] = [[1.0, np.inf, 3.0], [np.nan, 2.0, -np.nan]]       # NaN sorts above infinity; equal payloads: the earlier
+    dy[0, 2] = [[-0.0, 0.0, -0.0], [0.0, 0.0, 0.0]]               # all zeros of either sign: position 0
+    dy[0, 3] = [[-0.0, 0.0, 1e-300], [0.0, -1e-300, 0.0]]         # equal magnitudes of opposite sign: the earlier
+    dy[0, 4] = [[5.0, -7.0, 7.0], [1.0, 2.0, 3.0]]
+    dy[0, 5] = [[1.0, 2.0, 3.0], [4.0, 5.0, np.float64("nan")]]
+    idx, s, _ = oracle.top1_select(dy)
+    assert idx[0].tolist() == [1, 3, 0, 2, 1, 5]
+    assert np.isnan(s[0, 0]) and np.isnan(s[0, 1]) and s[0, 2] == 0 and s[0, 4] == 11.0      # the sum propagates as IEEE does
+    # for finite inputs the order is the order of |v|: same answer as numpy's first arg max of |v|
+    rng = np.random.default_rng(77)
+    d = rng.standard_normal((3, 4, 5, 6)).astype(np.float32).astype(np.float64)
+    want = np.argmax(np.abs(d).reshape(3, 4, -1), axis=2)
+    np.testing.assert_array_equal(oracle.top1_select(d)[0], want)
+
+
+# ---- top-k variant: pinned by k = 1, by the sparse list, by brute force, and by the constant-X case ----
+@pytest.mark.parametrize("g", GEOMS)
+def test_topk_with_k_one_is_algorithm_1(g):
+    x, dy = _rand(g, 30)
+    a, an = oracle.dw_topk(x, dy, g, 1, 0.5)
+    b, bn = oracle.dw_top1(x, dy, g, 0.5)
+    np.testing.assert_array_equal(a, b)
+    np.testing.assert_array_equal(an, bn)
+    np.testing.assert_array_equal(oracle.topk_select(dy, 1)[0][..., 0], oracle.top1_select(dy)[0])
+
+
+@pytest.mark.parametrize("topk", [2, 3, 5])
+@pytest.mark.parametrize("g", GEOMS[:3])
+def test_topk_equals_the_sparse_list_with_sum_over_k(g, topk):
+    x, dy = _rand(g, 31)
+    t = min(topk, g.p * g.q)
+    # brute-force selection: stable sort of positions by descending |v| (numpy), first t of each map
+    flat = dy.reshape(g.n, g.k, -1)
+    order = np.argsort(-np.abs(flat), axis=2, kind="stable")[..., :t]
+    idx, s, _ = oracle.topk_select(dy, topk)
+    np.testing.assert_array_equal(idx, order)
+    np.testing.assert_allclose(s, flat.sum(axis=2), rtol=0, atol=1e-12)
+    entries = [(n, k, int(j) // g.q, int(j) % g.q, float(flat[n, k].sum() / t))
+               for n in range(g.n) for k in range(g.k) for j in order[n, k]]
+    np.testing.assert_allclose(oracle.dw_topk(x, dy, g, topk, 0.25)[0], oracle.dw_sparse(x, entries, g, 0.25), rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("topk", [1, 2, 4, 9])
+def test_topk_is_exact_for_spatially_constant_x_without_padding(topk):
+    """Every patch is the same constant, so any k retained entries that add up to the map's sum give the exact gradient."""
+    g = oracle.Shape(3, 4, 7, 7, 5, 3, 3, 2, 2, 0, 0)
+    rng = np.random.default_rng(32)
+    x = np.broadcast_to(rng.standard_normal((g.n, g.c, 1, 1)), (g.n, g.c, g.h, g.w)).copy()
+    dy = rng.standard_normal((g.n, g.k, g.p, g.q))
+    np.testing.assert_allclose(oracle.dw_topk(x, dy, g, topk)[0], oracle.dw_exact(x, dy, g)[0], rtol=0, atol=1e-12)
+
+
+def test_topk_keeping_every_position_of_a_constant_map_is_exact():
+    """k = P*Q with a map whose entries are all equal: each keeps sum/k = its own value, so top-k equals exact dW."""
+    g = oracle.Shape(2, 3, 6, 6, 4, 3, 3, 1, 1, 1, 1)
+    rng = np.random.default_rng(33)
+    x = rng.standard_normal((g.n, g.c, g.h, g.w))
+    dy = np.broadcast_to(rng.standard_normal((g.n, g.k, 1, 1)), (g.n, g.k, g.p, g.q)).copy()
+    np.testing.assert_allclose(oracle.dw_topk(x, dy, g, g.p * g.q)[0], oracle.dw_exact(x, dy, g)[0], rtol=0, atol=1e-12)
