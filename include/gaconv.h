@@ -44,9 +44,11 @@ typedef enum {
 typedef enum { GACONV_F32 = 0, GACONV_BF16 = 1 } gaconv_dtype_t;            /* of x and dy            */
 typedef enum { GACONV_X_NHWC = 0, GACONV_X_NCHW = 1 } gaconv_x_layout_t;    /* NHWC: Section 2.4     */
 typedef enum { GACONV_DY_NKPQ = 0 } gaconv_dy_layout_t;                     /* = N C_o H W           */
-typedef enum { GACONV_DW_KRSC = 0, GACONV_DW_KCRS = 1 } gaconv_dw_layout_t; /* KRSC = C_o K K C_i    */
+/* KRSC = C_o K K C_i (the layout of the paper's kernel, Section 2.4), KCRS = the frameworks' filter
+ * layout, RSCK = K K C_i C_o (the order in which Section 2.4 first writes df) */
+typedef enum { GACONV_DW_KRSC = 0, GACONV_DW_KCRS = 1, GACONV_DW_RSCK = 2 } gaconv_dw_layout_t;
 typedef enum { GACONV_METHOD_EXACT = -1, GACONV_METHOD_ZERO = 0, GACONV_METHOD_RANDOM = 1,
-               GACONV_METHOD_TOP1 = 2 } gaconv_method_t;
+               GACONV_METHOD_TOP1 = 2, GACONV_METHOD_TOPK = 3 } gaconv_method_t;
 /* arithmetic of the exact contraction */
 typedef enum {
     GACONV_MATH_DEFAULT = 0,   /* bf16 inputs: bf16 tensor cores, fp32 accumulate; fp32 inputs: fp32-accurate
@@ -67,11 +69,14 @@ typedef struct gaconv_conv_desc {
     int32_t  x_layout, dy_layout, dw_layout;
     int32_t  math;                     /* gaconv_math_t                                                   */
     int32_t  algo;                     /* gaconv_algo_t                                                   */
+    int32_t  topk;                     /* GACONV_METHOD_TOPK: entries retained per map, 1..GACONV_MAX_TOPK (else ignored) */
     float    alpha;                    /* dw = alpha * (...); 1 for parity, 1/128 in the paper's runs (Section 2.3) */
     float    rand_std;                 /* METHOD_RANDOM: standard deviation; the paper uses 1/128 (Section 2.2)     */
     void    *workspace;                /* device scratch prepared by gaconv_workspace_init                */
     size_t   workspace_bytes;
 } gaconv_conv_desc_t;
+
+#define GACONV_MAX_TOPK 16
 
 const char *gaconv_status_string(gaconv_status_t status);
 
@@ -119,6 +124,11 @@ gaconv_status_t gaconv_dw_exact(const void *x, const void *dy, float *dw,
 gaconv_status_t gaconv_dw_exact_static(const void *x, const void *dy, float *dw,
                                        const gaconv_conv_desc_t *desc, void *stream);
 size_t gaconv_static_scratch_bytes(void);
+/* gaconv_poll_async_status for the built-in array of gaconv_dw_exact_static on the current device (the
+ * paper has no counterpart): waits for `stream`, then GACONV_ERR_TIMEOUT if a kernel launched through
+ * gaconv_dw_exact_static gave up on a bounded wait since the last poll (clears the flag), else GACONV_OK.
+ * Before the first gaconv_dw_exact_static call on the device it returns GACONV_OK.  Allocates nothing. */
+gaconv_status_t gaconv_poll_async_status_static(void *stream);
 
 /* Approximated filter gradient, Section 2:
  *   GACONV_METHOD_ZERO   (2.1)  dw = +0.
@@ -129,7 +139,11 @@ size_t gaconv_static_scratch_bytes(void);
  *   GACONV_METHOD_TOP1   (2.3, Algorithm 1)  for every (n,k): keep only the largest-magnitude entry of
  *        dy[n,k,:,:] (lowest p*Q+q among equals), replace it by the signed sum of the map, and take
  *        the exact filter gradient of that sparse tensor.
- * `seed` is ignored by ZERO and TOP1. */
+ *   GACONV_METHOD_TOPK   (2.3: the method "can be modified" to keep the k largest magnitudes, with an
+ *        adjusted scale that the paper leaves open)  keep the desc->topk largest-magnitude entries of every
+ *        map (equal magnitudes: lower p*Q+q first), give each of them sum/topk, and take the exact filter
+ *        gradient of that sparse tensor.  topk = 1 is TOP1; topk is clamped to P*Q.
+ * `seed` is ignored by ZERO, TOP1 and TOPK. */
 gaconv_status_t gaconv_dw_approx(int32_t method, const void *x, const void *dy, float *dw,
                                  const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
 
@@ -139,6 +153,11 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void *x, const void *dy, 
  * to in_dtype, at the retained position and zero elsewhere.  Needs no workspace. */
 gaconv_status_t gaconv_approx_select(const void *dy, int32_t *idx, float *sum, void *dy_sparse,
                                      const gaconv_conv_desc_t *desc, void *stream);
+
+/* Selection step of the top-k variant, for inspection: idx[(n*K+k)*t + i] = position of the i-th retained
+ * entry of dy[n,k,:,:] in order of selection (t = min(desc->topk, P*Q)), sum[n*K+k] = signed sum of the map. */
+gaconv_status_t gaconv_approx_select_topk(const void *dy, int32_t *idx, float *sum,
+                                          const gaconv_conv_desc_t *desc, void *stream);
 
 /* Same operation as gaconv_dw_exact / gaconv_dw_approx (method as above, GACONV_METHOD_EXACT for
  * exact) with HOST inputs and output: copies x_host and dy_host into the caller's device staging

@@ -21,8 +21,9 @@ ERR_NULL_POINTER, ERR_BAD_DESC, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_WORKSPACE_T
 F32, BF16 = 0, 1
 X_NHWC, X_NCHW = 0, 1
 DY_NKPQ = 0
-DW_KRSC, DW_KCRS = 0, 1
-METHOD_EXACT, METHOD_ZERO, METHOD_RANDOM, METHOD_TOP1 = -1, 0, 1, 2
+DW_KRSC, DW_KCRS, DW_RSCK = 0, 1, 2
+METHOD_EXACT, METHOD_ZERO, METHOD_RANDOM, METHOD_TOP1, METHOD_TOPK = -1, 0, 1, 2, 3
+MAX_TOPK = 16
 MATH_DEFAULT, MATH_TF32 = 0, 1
 ALGO_AUTO, ALGO_DIRECT, ALGO_TENSOR = 0, 1, 2
 SCHED_EVERY_4TH_LAYER, SCHED_ALT_LAYER_ALT_BATCH, SCHED_ALL_LAYERS_EVERY_4TH_BATCH, SCHED_LAYER2_ALT_BATCH, \
@@ -32,14 +33,14 @@ EXPORTS = [
     "gaconv_status_string", "gaconv_launch_count", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
     "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_poll_async_status",
     "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_destroy",
-    "gaconv_dw_exact_static", "gaconv_static_scratch_bytes",
+    "gaconv_dw_exact_static", "gaconv_static_scratch_bytes", "gaconv_poll_async_status_static", "gaconv_approx_select_topk",
 ]
 
 
 class ConvDesc(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32)] + \
         [(f, ctypes.c_int32) for f in ("n", "c", "h", "w", "k", "r", "s", "stride_h", "stride_w", "pad_h", "pad_w",
-                                       "in_dtype", "x_layout", "dy_layout", "dw_layout", "math", "algo")] + \
+                                       "in_dtype", "x_layout", "dy_layout", "dw_layout", "math", "algo", "topk")] + \
         [("alpha", ctypes.c_float), ("rand_std", ctypes.c_float),
          ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
@@ -78,6 +79,8 @@ def load():
     lib.gaconv_approx_select.argtypes = [vp, vp, vp, vp, dp, vp]
     lib.gaconv_dw_from_host.argtypes = [i32, vp, vp, vp, vp, vp, vp, dp, u64, vp]
     lib.gaconv_poll_async_status.argtypes = [dp, vp]
+    lib.gaconv_poll_async_status_static.argtypes = [vp]
+    lib.gaconv_approx_select_topk.argtypes = [vp, vp, vp, dp, vp]
     lib.gaconv_schedule_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, ctypes.c_double, u64]
     lib.gaconv_schedule_method.argtypes = [vp, i32, ctypes.c_int64]
     lib.gaconv_schedule_method.restype = i32
@@ -118,7 +121,7 @@ def _stream(stream):
 
 
 def make_desc(layer: ConvLayer, dtype: torch.dtype, *, x_layout=X_NHWC, dw_layout=DW_KRSC, alpha=1.0,
-              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO) -> ConvDesc:
+              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO, topk=1) -> ConvDesc:
     d = ConvDesc()
     d.struct_size = ctypes.sizeof(ConvDesc)
     d.n, d.c, d.h, d.w, d.k, d.r, d.s = layer.n, layer.c, layer.h, layer.w, layer.k, layer.r, layer.s
@@ -126,7 +129,7 @@ def make_desc(layer: ConvLayer, dtype: torch.dtype, *, x_layout=X_NHWC, dw_layou
     d.pad_h = d.pad_w = layer.pad
     d.in_dtype = BF16 if dtype == torch.bfloat16 else F32
     d.x_layout, d.dy_layout, d.dw_layout = x_layout, DY_NKPQ, dw_layout
-    d.math, d.algo = math, algo
+    d.math, d.algo, d.topk = math, algo, topk
     d.alpha, d.rand_std = alpha, rand_std
     d.workspace, d.workspace_bytes = None, 0
     return d
@@ -142,10 +145,11 @@ def gaconv_workspace_init(workspace, nbytes: int, stream=None):
     _check(load().gaconv_workspace_init(_ptr(workspace), nbytes, _stream(stream)), "gaconv_workspace_init")
 
 
-def attach_workspace(desc: ConvDesc, methods=(METHOD_EXACT, METHOD_TOP1), device="cuda") -> torch.Tensor:
+def attach_workspace(desc: ConvDesc, methods=(METHOD_EXACT, METHOD_TOP1, METHOD_TOPK), device="cuda") -> torch.Tensor:
     """Allocate (with torch) and initialise a workspace large enough for `methods`; returns the tensor
     that owns the memory -- keep it alive as long as the descriptor is used."""
-    need = max(gaconv_workspace_size(desc, m) for m in methods)
+    usable = [m for m in methods if m != METHOD_TOPK or 1 <= desc.topk <= MAX_TOPK]
+    need = max(gaconv_workspace_size(desc, m) for m in usable)
     ws = torch.empty(need, dtype=torch.uint8, device=device)
     gaconv_workspace_init(ws, need)
     desc.workspace, desc.workspace_bytes = ws.data_ptr(), need
@@ -178,6 +182,11 @@ def gaconv_approx_select(dy, idx, sum_, dy_sparse, desc: ConvDesc, stream=None):
                                        _stream(stream)), "gaconv_approx_select")
 
 
+def gaconv_approx_select_topk(dy, idx, sum_, desc: ConvDesc, stream=None):
+    _check(load().gaconv_approx_select_topk(_ptr(dy), _ptr(idx), _ptr(sum_), ctypes.byref(desc), _stream(stream)),
+           "gaconv_approx_select_topk")
+
+
 def gaconv_dw_from_host(method: int, x_host, dy_host, dw_host, x_dev, dy_dev, dw_dev, desc: ConvDesc, seed: int = 0,
                         stream=None):
     _check(load().gaconv_dw_from_host(method, _ptr(x_host), _ptr(dy_host), _ptr(dw_host), _ptr(x_dev), _ptr(dy_dev),
@@ -186,6 +195,10 @@ def gaconv_dw_from_host(method: int, x_host, dy_host, dw_host, x_dev, dy_dev, dw
 
 def gaconv_poll_async_status(desc: ConvDesc, stream=None) -> int:
     return load().gaconv_poll_async_status(ctypes.byref(desc), _stream(stream))
+
+
+def gaconv_poll_async_status_static(stream=None) -> int:
+    return load().gaconv_poll_async_status_static(_stream(stream))
 
 
 class Schedule:

@@ -25,7 +25,7 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     if (d->in_dtype != GACONV_F32 && d->in_dtype != GACONV_BF16) return GACONV_ERR_BAD_DESC;
     if (d->x_layout != GACONV_X_NHWC && d->x_layout != GACONV_X_NCHW) return GACONV_ERR_BAD_DESC;
     if (d->dy_layout != GACONV_DY_NKPQ) return GACONV_ERR_BAD_DESC;
-    if (d->dw_layout != GACONV_DW_KRSC && d->dw_layout != GACONV_DW_KCRS) return GACONV_ERR_BAD_DESC;
+    if (d->dw_layout != GACONV_DW_KRSC && d->dw_layout != GACONV_DW_KCRS && d->dw_layout != GACONV_DW_RSCK) return GACONV_ERR_BAD_DESC;
     if (d->math != GACONV_MATH_DEFAULT && d->math != GACONV_MATH_TF32) return GACONV_ERR_BAD_DESC;
     if (d->algo < GACONV_ALGO_AUTO || d->algo > GACONV_ALGO_TENSOR) return GACONV_ERR_BAD_DESC;
     g->n = d->n; g->c = d->c; g->h = d->h; g->w = d->w; g->k = d->k; g->r = d->r; g->s = d->s;
@@ -42,8 +42,10 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     }
     if (d->dw_layout == GACONV_DW_KRSC) {
         g->ws_c = 1; g->ws_s = d->c; g->ws_r = (long long)d->s * d->c; g->ws_k = (long long)d->r * d->s * d->c;
-    } else {
+    } else if (d->dw_layout == GACONV_DW_KCRS) {
         g->ws_s = 1; g->ws_r = d->s; g->ws_c = (long long)d->r * d->s; g->ws_k = (long long)d->c * d->r * d->s;
+    } else {
+        g->ws_k = 1; g->ws_c = d->k; g->ws_s = (long long)d->c * d->k; g->ws_r = (long long)d->s * d->c * d->k;
     }
     g->bf16 = d->in_dtype == GACONV_BF16;
     g->alpha = d->alpha;
@@ -91,6 +93,27 @@ ExactLayout exact_layout(const Geom& g)
     if (L.stem_ok && L.sp.partial_bytes > partial) partial = L.sp.partial_bytes;
     L.scratch_off = align_up(L.partial_off + partial, 256);
     L.total = align_up(L.scratch_off + (L.tc_ok ? L.tp.scratch_bytes : 0), 256);
+    return L;
+}
+
+// entries retained per map by the top-k method: desc->topk clamped to the map size; 0 = invalid
+int topk_of(const gaconv_conv_desc_t* d, const Geom& g)
+{
+    if (d->topk < 1 || d->topk > GACONV_MAX_TOPK) return 0;
+    const long long pq = (long long)g.p * g.q;
+    return d->topk < pq ? d->topk : (int)pq;
+}
+
+struct TopkLayout { size_t idx_off, sum_off, partial_off, total; GatherPlan gp; };
+TopkLayout topk_layout(const Geom& g, int topk)
+{
+    TopkLayout L;
+    L.gp = plan_gather(g);
+    const size_t maps = (size_t)g.n * g.k;
+    L.idx_off = kWsDataOffset;
+    L.sum_off = align_up(L.idx_off + maps * topk * sizeof(int32_t), 256);
+    L.partial_off = align_up(L.sum_off + maps * sizeof(float), 256);
+    L.total = align_up(L.partial_off + L.gp.partial_bytes, 256);
     return L;
 }
 
@@ -147,6 +170,12 @@ gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t me
     switch (method) {
         case GACONV_METHOD_EXACT: *bytes = exact_layout(g).total; return GACONV_OK;
         case GACONV_METHOD_TOP1: *bytes = top1_layout(g).total; return GACONV_OK;
+        case GACONV_METHOD_TOPK: {
+            const int t = topk_of(desc, g);
+            if (t < 1) return GACONV_ERR_BAD_DESC;
+            *bytes = topk_layout(g, t).total;
+            return GACONV_OK;
+        }
         case GACONV_METHOD_ZERO:
         case GACONV_METHOD_RANDOM: *bytes = kWsDataOffset; return GACONV_OK;
     }
@@ -212,9 +241,25 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     if (method == GACONV_METHOD_ZERO) return launch_zero(dw, count, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     if (method == GACONV_METHOD_RANDOM)
         return launch_random(dw, g, seed, desc->rand_std, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
-    if (method != GACONV_METHOD_TOP1) return GACONV_ERR_BAD_DESC;
+    if (method != GACONV_METHOD_TOP1 && method != GACONV_METHOD_TOPK) return GACONV_ERR_BAD_DESC;
     if (x == nullptr || dy == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy)) return GACONV_ERR_MISALIGNED;
+    if (method == GACONV_METHOD_TOPK) {
+        // selection of the topk largest magnitudes per map, then the patch accumulation over the retained entries
+        const int t = topk_of(desc, g);
+        if (t < 1) return GACONV_ERR_BAD_DESC;
+        const TopkLayout L = topk_layout(g, t);
+        st = check_ws(desc, L.total);
+        if (st != GACONV_OK) return st;
+        char* ws = static_cast<char*>(desc->workspace);
+        int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx_off);
+        float* sum = reinterpret_cast<float*>(ws + L.sum_off);
+        if (launch_select_topk(dy, idx, sum, g, t, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        if (launch_gather(x, idx, sum, dw, reinterpret_cast<float*>(ws + L.partial_off),
+                          reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, t, cs) != cudaSuccess)
+            return GACONV_ERR_CUDA;
+        return GACONV_OK;
+    }
     const Top1Layout L = top1_layout(g);
     st = check_ws(desc, L.total);       // required by every route, so that behaviour does not depend on the kernel picked
     if (st != GACONV_OK) return st;
@@ -232,7 +277,7 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
         return launch_top1_fused(x, dy, dw, g, cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
     if (launch_select(dy, idx, sum, nullptr, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
     if (launch_gather(x, idx, sum, dw, reinterpret_cast<float*>(ws + L.partial_off),
-                      reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, cs) != cudaSuccess)
+                      reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, 1, cs) != cudaSuccess)
         return GACONV_ERR_CUDA;
     return GACONV_OK;
 }
@@ -249,6 +294,18 @@ gaconv_status_t gaconv_approx_select(const void* dy, int32_t* idx, float* sum, v
                                                                                                          : GACONV_ERR_CUDA;
 }
 
+gaconv_status_t gaconv_approx_select_topk(const void* dy, int32_t* idx, float* sum, const gaconv_conv_desc_t* desc, void* stream)
+{
+    Geom g;
+    gaconv_status_t st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    if (dy == nullptr || idx == nullptr || sum == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (!aligned16(dy) || !aligned16(idx) || !aligned16(sum)) return GACONV_ERR_MISALIGNED;
+    const int t = topk_of(desc, g);
+    if (t < 1) return GACONV_ERR_BAD_DESC;
+    return launch_select_topk(dy, idx, sum, g, t, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+}
+
 gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
                                     void* x_dev, void* dy_dev, float* dw_dev, const gaconv_conv_desc_t* desc,
                                     uint64_t seed, void* stream)
@@ -258,9 +315,24 @@ gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const vo
     if (st != GACONV_OK) return st;
     if (dw_host == nullptr || dw_dev == nullptr) return GACONV_ERR_NULL_POINTER;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    const bool needs_inputs = method == GACONV_METHOD_EXACT || method == GACONV_METHOD_TOP1;
+    const bool needs_inputs = method == GACONV_METHOD_EXACT || method == GACONV_METHOD_TOP1 || method == GACONV_METHOD_TOPK;
+    // everything the compute call would reject is rejected here, before the first copy is enqueued
+    if (method < GACONV_METHOD_EXACT || method > GACONV_METHOD_TOPK) return GACONV_ERR_BAD_DESC;
+    if (!aligned16(dw_dev)) return GACONV_ERR_MISALIGNED;
     if (needs_inputs) {
         if (x_host == nullptr || dy_host == nullptr || x_dev == nullptr || dy_dev == nullptr) return GACONV_ERR_NULL_POINTER;
+        if (!aligned16(x_dev) || !aligned16(dy_dev)) return GACONV_ERR_MISALIGNED;
+        if (method == GACONV_METHOD_EXACT && desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
+        size_t need = 0;
+        st = gaconv_workspace_size(desc, method, &need);
+        if (st != GACONV_OK) return st;
+        st = check_ws(desc, need);
+        if (st != GACONV_OK) return st;
+        if (method == GACONV_METHOD_EXACT) {
+            const ExactLayout L = exact_layout(g);
+            if (desc->math == GACONV_MATH_TF32 && !direct_mma_supported(g, L.dp)) return GACONV_ERR_UNSUPPORTED;
+            if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
+        }
         const size_t eb = g.bf16 ? 2 : 4;
         if (cudaMemcpyAsync(x_dev, x_host, (size_t)g.n * g.c * g.h * g.w * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
             cudaMemcpyAsync(dy_dev, dy_host, (size_t)g.n * g.k * g.p * g.q * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess)
@@ -296,7 +368,8 @@ gaconv_status_t gaconv_schedule_create(gaconv_schedule_t** out, int32_t num_laye
     *out = nullptr;
     if (num_layers < 1 || num_layers > (1 << 20)) return GACONV_ERR_BAD_DESC;
     if (kind < GACONV_SCHED_EVERY_4TH_LAYER || kind > GACONV_SCHED_SEEDED_FRACTION_ALT_BATCH) return GACONV_ERR_BAD_DESC;
-    if (method != GACONV_METHOD_ZERO && method != GACONV_METHOD_RANDOM && method != GACONV_METHOD_TOP1) return GACONV_ERR_BAD_DESC;
+    if (method != GACONV_METHOD_ZERO && method != GACONV_METHOD_RANDOM && method != GACONV_METHOD_TOP1 && method != GACONV_METHOD_TOPK)
+        return GACONV_ERR_BAD_DESC;
     if (!(fraction >= 0.0 && fraction <= 1.0)) return GACONV_ERR_BAD_DESC;
     gaconv_schedule* s = new (std::nothrow) gaconv_schedule{num_layers, kind, method, fraction, seed, nullptr};
     if (s == nullptr) return GACONV_ERR_BAD_DESC;

@@ -1,10 +1,9 @@
-// Exact filter gradient on the warp-level tensor-core path.  fp32 inputs (the main use): mma.sync m16n8k8,
+// Exact filter gradient of fp32 inputs on the warp-level tensor-core path: mma.sync m16n8k8,
 // TF32 operands, fp32 accumulate, with the operands split so that fp32 accuracy is kept:
 //   x = big + small,  big = tf32(x) (by truncation),  small = tf32(x - big)
 //   a*b ~= big_a*big_b + big_a*small_b + small_a*big_b            ("3xTF32": error ~ 2^-21 per product)
 // One pass (big*big only) is the opt-in GACONV_MATH_TF32 mode: operands cut to 10 mantissa bits.
-// bf16 inputs run one pass of m16n8k16; the tcgen05 kernel is faster wherever it tiles the shape (measured
-// 11-12 us against 13-14 us on the 16- and 32-channel ResNet-20 layers), so this serves the remaining shapes.
+// (bf16 inputs take the tcgen05 kernel, which measured faster wherever both tile the shape, or the FP32 pipes.)
 //
 //   dW[k,c,r,s] = alpha * sum_{n,p,q} Xz[n,c,p*st+r-pad,q*st+s-pad] * dY[n,k,p,q]              (Section 2.4)
 //
@@ -26,9 +25,7 @@ namespace {
 
 constexpr int kThreads = 128, kWarps = 4, TK = 16, TC = 16;
 
-
-// BF16: bf16 inputs on m16n8k16 (one pass, products exact in fp32; 64 pixels per dY box, 16 per k-step).
-template <int R, int S, bool THREE_PASS, bool BF16>
+template <int R, int S, bool THREE_PASS>
 __global__ void __launch_bounds__(kThreads)
 direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ status,
                   const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
@@ -47,7 +44,7 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
 
     const int npx = pl.bp * pl.bq;                       // a multiple of 32; bq == Q, a multiple of 8
     const int win_h = (pl.bp - 1) * g.stride_h + R, win_w = (pl.bq - 1) * g.stride_w + S;
-    constexpr int EB = BF16 ? 2 : 4, BOXPX = BF16 ? 64 : 32, KPX = BF16 ? 16 : 8;
+    constexpr int EB = 4, BOXPX = 32, KPX = 8;
     const int dy_bytes = npx / BOXPX * 2048;             // [boxes][16 k][128-byte swizzled rows]
     const int x_bytes = win_h * win_w * TC * EB;         // [row][col][16 c]
     const int stage_bytes = (dy_bytes + x_bytes + 1023) & ~1023;
@@ -91,38 +88,10 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
         __syncthreads();
         if (s_fail) { if (threadIdx.x == 0) atomicOr(status, 1u); break; }   // uniform exit
         const uint8_t* s_dy = smem + stage * stage_bytes;
-        const float* s_x = reinterpret_cast<const float*>(s_dy + dy_bytes);   // bf16 inputs: reinterpreted below
+        const float* s_x = reinterpret_cast<const float*>(s_dy + dy_bytes);
 
         for (int ks = SPLIT_TAPS ? 0 : warp; ks < npx / KPX; ks += SPLIT_TAPS ? 1 : kWarps) {
             const int px0 = ks * KPX;
-            if constexpr (BF16) {
-                // A: dY[k = gq (+8)][px0 + 2*tq, +1 (+8, +9)], two bf16 per register
-                uint32_t a[4];
-                const uint8_t* box = s_dy + (px0 >> 6) * 2048;
-                const int ch0 = (px0 & 63) >> 3;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = gq + (i & 1) * 8, ch = ch0 + (i >> 1);
-                    a[i] = *reinterpret_cast<const uint32_t*>(box + row * 128 + ((ch ^ (row & 7)) << 4) + tq * 4);
-                }
-                const int pp = px0 / pl.bq, qq = px0 - pp * pl.bq;
-                const unsigned short* xrow = reinterpret_cast<const unsigned short*>(s_x) + ((pp * g.stride_h) * win_w + (qq + 2 * tq) * g.stride_w) * TC + gq;
-                const int px1 = g.stride_w * TC, px8 = 8 * px1;
-#pragma unroll
-                for (int i = 0; i < TPW; ++i) {
-                    const int tap = tap_lo + i;
-                    if (SPLIT_TAPS && tap >= TAPS) break;
-                    const int r = SPLIT_TAPS ? tap / S : i / S, s = SPLIT_TAPS ? tap % S : i % S;
-                    const unsigned short* xt = xrow + (r * win_w + s) * TC;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t b0 = (uint32_t)xt[h * 8] | ((uint32_t)xt[h * 8 + px1] << 16);
-                        const uint32_t b1 = (uint32_t)xt[h * 8 + px8] | ((uint32_t)xt[h * 8 + px8 + px1] << 16);
-                        mma_bf16(acc[i * 2 + h], a, b0, b1);
-                    }
-                }
-                continue;
-            }
             // ---- A fragment: dY[k = gq (+8)][px0 + tq (+4)], from the swizzled box ----
             uint32_t a_big[4], a_small[4];
             {
@@ -193,10 +162,10 @@ direct_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t*
 
 bool direct_mma_supported(const Geom& g, const DirectPlan& pl)
 {
-    if (g.xs_c != 1 || g.c % (g.bf16 ? 8 : 4) != 0 || g.c < 8) return false;
+    if (g.bf16 || g.xs_c != 1 || g.c % 4 != 0 || g.c < 8) return false;
     if (g.r != g.s || (g.r != 1 && g.r != 3 && g.r != 5)) return false;
     const int npx = pl.bp * pl.bq, pq = g.p * g.q;
-    const int boxpx = g.bf16 ? 64 : 32, kpx = g.bf16 ? 16 : 8;
+    const int boxpx = 32, kpx = 8;
     if (pl.bq != g.q || g.q % kpx != 0 || g.p % pl.bp != 0 || npx % boxpx != 0 || npx > 256 || pq % 8 != 0) return false;
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
     if (win_h > 256 || win_w > 256) return false;
@@ -210,8 +179,8 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     const int win_h = (pl.bp - 1) * g.stride_h + g.r, win_w = (pl.bq - 1) * g.stride_w + g.s;
     CUtensorMap map_dy, map_x;
     cuuint64_t d3[3] = {(cuuint64_t)pq, (cuuint64_t)g.k, (cuuint64_t)g.n};
-    const int eb = g.bf16 ? 2 : 4, boxpx = g.bf16 ? 64 : 32;
-    const CUtensorMapDataType dt = g.bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    const int eb = 4, boxpx = 32;
+    const CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     cuuint64_t s3[2] = {(cuuint64_t)pq * eb, (cuuint64_t)g.k * pq * eb};
     cuuint32_t b3[3] = {(cuuint32_t)boxpx, (cuuint32_t)TK, 1}, e3[3] = {1, 1, 1};
     cuuint64_t d4[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
@@ -229,8 +198,8 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     dim3 grid(pl.tiles_k * pl.tiles_c, pl.splits);
     cudaError_t launch_err = cudaErrorInvalidValue;
 #define GACONV_MMA_CASE(RR, TP)                                                                                          \
-    if (g.r == RR && three_pass == TP && !g.bf16) {                                                                      \
-        auto kern = direct_mma_kernel<RR, RR, TP, false>;                                                                       \
+    if (g.r == RR && three_pass == TP) {                                                                                 \
+        auto kern = direct_mma_kernel<RR, RR, TP>;                                                                       \
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
         launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), dw, partial, status, map_dy, map_x, g, pl); \
     }
@@ -241,16 +210,6 @@ cudaError_t launch_direct_mma(const void* x, const void* dy, float* dw, float* p
     GACONV_MMA_CASE(5, true)
     GACONV_MMA_CASE(5, false)
 #undef GACONV_MMA_CASE
-#define GACONV_MMA_BF16_CASE(RR)                                                                                         \
-    if (g.r == RR && g.bf16) {                                                                                           \
-        auto kern = direct_mma_kernel<RR, RR, false, true>;                                                             \
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
-        launch_err = launch_kernel(kern, grid, dim3(kThreads), smem, stream, dim3(1, 1, 1), dw, partial, status, map_dy, map_x, g, pl); \
-    }
-    GACONV_MMA_BF16_CASE(1)
-    GACONV_MMA_BF16_CASE(3)
-    GACONV_MMA_BF16_CASE(5)
-#undef GACONV_MMA_BF16_CASE
     note_launch();
     if (launch_err != cudaSuccess) return launch_err;
     if (pl.splits > 1) return reduce_splits(partial, dw, (size_t)g.k * g.c * g.r * g.s, pl.splits, g.alpha, stream);

@@ -79,7 +79,9 @@ struct GatherPlan {
 };
 GatherPlan plan_gather(const Geom& g);
 cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, float* dw, float* partial,
-                          uint32_t* counters, const Geom& g, const GatherPlan& plan, cudaStream_t stream);
+                          uint32_t* counters, const Geom& g, const GatherPlan& plan, int topk, cudaStream_t stream);
+// selection of the top-k variant: idx[map][topk] in order of selection, sum[map]
+cudaError_t launch_select_topk(const void* dy, int32_t* idx, float* sum, const Geom& g, int topk, cudaStream_t stream);
 
 // ---- Algorithm 1 in one launch (selection + patch accumulate + cluster reduction) ----
 bool top1_fused_supported(const Geom& g);

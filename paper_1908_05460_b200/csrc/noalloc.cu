@@ -48,6 +48,29 @@ extern "C" {
 
 size_t gaconv_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
+// The status word of the built-in array (its first four bytes) is where a kernel launched through
+// gaconv_dw_exact_static records that it gave up on a bounded wait.  Read and cleared like the
+// caller-owned workspace's word; no allocation, and nothing to do before the array's first use.
+gaconv_status_t gaconv_poll_async_status_static(void* stream)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return GACONV_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_setup_mutex);
+        scratch = g_scratch_ptr[dev];
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (scratch == nullptr) return cudaStreamSynchronize(cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    if (word == 0) return GACONV_OK;
+    if (cudaMemsetAsync(scratch, 0, sizeof(word), cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    return GACONV_ERR_TIMEOUT;
+}
+
 gaconv_status_t gaconv_dw_exact_static(const void* x, const void* dy, float* dw, const gaconv_conv_desc_t* desc, void* stream)
 {
     if (desc == nullptr) return GACONV_ERR_NULL_POINTER;

@@ -149,6 +149,41 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
     }
 }
 
+// Selection of the top-k variant: one warp per map.  Round t picks the largest key below the key picked in
+// round t-1, where key = (bit pattern of |v|, complement of the position): keys are distinct, larger magnitude
+// first and, among equal magnitudes, the lower position first -- the order the single arg-max uses.
+template <typename T>
+__global__ void __launch_bounds__(256)
+select_topk_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __restrict__ sum, long long num_maps, int pq, int topk)
+{
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
+    const int lane = threadIdx.x & 31;
+    const long long m = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (m >= num_maps) return;
+    const T* map = dy + m * (long long)pq;
+    unsigned long long prev = ~0ull;
+    float total = 0.0f;
+    for (int t = 0; t < topk; ++t) {
+        unsigned long long best = 0ull;
+        for (int j = lane; j < pq; j += 32) {
+            Scan sc{-1, 0, 0.0f};
+            Elem<T>::visit1(map, j, sc);
+            const unsigned long long key = ((unsigned long long)(unsigned)(sc.best_mag + 1) << 32) | (0xffffffffu - (unsigned)j);
+            if (key < prev && key > best) best = key;
+            if (t == 0) total += sc.sum;
+        }
+        for (int off = 16; off > 0; off >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, off);
+            best = other > best ? other : best;
+        }
+        if (lane == 0) idx[m * topk + t] = (int)(0xffffffffu - (unsigned)(best & 0xffffffffu));
+        prev = best;
+    }
+    for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+    if (lane == 0) sum[m] = total;
+}
+
 // four consecutive elements, raw (16-byte load for fp32, 8-byte load for bf16), and their values as floats
 struct Raw4 { uint32_t w[4]; };
 __device__ __forceinline__ Raw4 ld4_raw(const float* p) {
@@ -288,31 +323,33 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
 }
 
 // grid (chunks, K).  Each CTA owns the images [chunk*ipc, (chunk+1)*ipc) of one output channel and
-// accumulates their patches in image order; the last CTA of a channel to finish adds the per-chunk
-// partials in chunk order (fixed order => reproducible) and writes dW.
+// accumulates their patches in image order (topk retained entries per map, each weighted sum/topk; topk = 1
+// is Algorithm 1); the last CTA of a channel to finish adds the per-chunk partials in chunk order (fixed
+// order => reproducible) and writes dW.
 template <typename T>
 __global__ void __launch_bounds__(256)
 gather_kernel(const T* __restrict__ x, const int32_t* __restrict__ idx, const float* __restrict__ sum,
               float* __restrict__ dw, float* __restrict__ partial, uint32_t* __restrict__ counters, Geom g,
-              int chunks, int ipc)
+              int chunks, int ipc, int topk)
 {
     pdl_release_next_grid();
     pdl_wait_prior_grid();
     extern __shared__ int smem_i[];
-    int* s_h0 = smem_i;                       // top-left input row of each image's patch
-    int* s_w0 = smem_i + ipc;
-    float* s_sum = reinterpret_cast<float*>(smem_i + 2 * ipc);
+    int* s_h0 = smem_i;                       // top-left input row of each retained entry's patch, [image][topk]
+    int* s_w0 = smem_i + ipc * topk;
+    float* s_sum = reinterpret_cast<float*>(smem_i + 2 * ipc * topk);   // [image]: sum / topk
     __shared__ bool s_last;
 
     const int k = blockIdx.y, chunk = blockIdx.x;
     const int n0 = chunk * ipc;
     const int cnt = min(ipc, g.n - n0);
-    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    for (int it = threadIdx.x; it < cnt * topk; it += blockDim.x) {
+        const int i = it / topk;
         const long long m = (long long)(n0 + i) * g.k + k;
-        const int j = idx[m];
-        s_h0[i] = (j / g.q) * g.stride_h - g.pad_h;
-        s_w0[i] = (j % g.q) * g.stride_w - g.pad_w;
-        s_sum[i] = sum[m];
+        const int j = idx[m * topk + (it - i * topk)];
+        s_h0[it] = (j / g.q) * g.stride_h - g.pad_h;
+        s_w0[it] = (j % g.q) * g.stride_w - g.pad_w;
+        if (it == i * topk) s_sum[i] = sum[m] / (float)topk;
     }
     __syncthreads();
 
@@ -321,11 +358,12 @@ gather_kernel(const T* __restrict__ x, const int32_t* __restrict__ idx, const fl
     for (int e = threadIdx.x; e < rsc; e += blockDim.x) {
         const int c = e % g.c, rs = e / g.c, s = rs % g.s, r = rs / g.s;
         float acc = 0.0f;
-        for (int i = 0; i < cnt; ++i) {
-            const int hh = s_h0[i] + r, ww = s_w0[i] + s;
-            if (hh >= 0 && hh < g.h && ww >= 0 && ww < g.w)
-                acc = fmaf(s_sum[i], ldf(x + (n0 + i) * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w), acc);
-        }
+        for (int i = 0; i < cnt; ++i)
+            for (int t = 0; t < topk; ++t) {
+                const int hh = s_h0[i * topk + t] + r, ww = s_w0[i * topk + t] + s;
+                if (hh >= 0 && hh < g.h && ww >= 0 && ww < g.w)
+                    acc = fmaf(s_sum[i], ldf(x + (n0 + i) * g.xs_n + c * g.xs_c + hh * g.xs_h + ww * g.xs_w), acc);
+            }
         if (chunks == 1) dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * acc;
         else part[e] = acc;
     }
@@ -386,6 +424,16 @@ cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_spa
     return cudaGetLastError();
 }
 
+cudaError_t launch_select_topk(const void* dy, int32_t* idx, float* sum, const Geom& g, int topk, cudaStream_t stream)
+{
+    const long long maps = (long long)g.n * g.k;
+    const unsigned grid = (unsigned)((maps + 7) / 8);
+    if (g.bf16) select_topk_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(dy), idx, sum, maps, g.p * g.q, topk);
+    else        select_topk_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(dy), idx, sum, maps, g.p * g.q, topk);
+    note_launch();
+    return cudaGetLastError();
+}
+
 GatherPlan plan_gather(const Geom& g)
 {
     GatherPlan p;
@@ -402,16 +450,17 @@ GatherPlan plan_gather(const Geom& g)
 }
 
 cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, float* dw, float* partial,
-                          uint32_t* counters, const Geom& g, const GatherPlan& plan, cudaStream_t stream)
+                          uint32_t* counters, const Geom& g, const GatherPlan& plan, int topk, cudaStream_t stream)
 {
     dim3 grid(plan.chunks, g.k);
-    const size_t smem = (size_t)plan.imgs_per_chunk * 12;
+    const size_t smem = (size_t)plan.imgs_per_chunk * (8 * topk + 4);
+    if (smem > 48 * 1024) return cudaErrorInvalidValue;
     if (g.bf16)
         gather_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), idx, sum, dw,
-                                                                   partial, counters, g, plan.chunks, plan.imgs_per_chunk);
+                                                                   partial, counters, g, plan.chunks, plan.imgs_per_chunk, topk);
     else
         gather_kernel<float><<<grid, 256, smem, stream>>>(static_cast<const float*>(x), idx, sum, dw, partial,
-                                                          counters, g, plan.chunks, plan.imgs_per_chunk);
+                                                          counters, g, plan.chunks, plan.imgs_per_chunk, topk);
     note_launch();
     return cudaGetLastError();
 }

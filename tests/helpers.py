@@ -27,14 +27,15 @@ class GpuLayer:
     """Device buffers + descriptor of one layer in the library's layouts."""
 
     def __init__(self, layer: ConvLayer, dtype, x_nchw: torch.Tensor, dy: torch.Tensor, *, x_layout=B.X_NHWC,
-                 dw_layout=B.DW_KRSC, alpha=1.0, rand_std=1.0 / 128, algo=B.ALGO_AUTO, math=B.MATH_DEFAULT):
+                 dw_layout=B.DW_KRSC, alpha=1.0, rand_std=1.0 / 128, algo=B.ALGO_AUTO, math=B.MATH_DEFAULT, topk=1):
         self.layer, self.dtype, self.dw_layout = layer, dtype, dw_layout
         self.x = (I.to_nhwc(x_nchw) if x_layout == B.X_NHWC else x_nchw.contiguous()).cuda()
         self.dy = dy.contiguous().cuda()
-        shape = (layer.k, layer.r, layer.s, layer.c) if dw_layout == B.DW_KRSC else (layer.k, layer.c, layer.r, layer.s)
+        shape = {B.DW_KRSC: (layer.k, layer.r, layer.s, layer.c), B.DW_KCRS: (layer.k, layer.c, layer.r, layer.s),
+                 B.DW_RSCK: (layer.r, layer.s, layer.c, layer.k)}[dw_layout]
         self.dw = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
         self.desc = B.make_desc(layer, dtype, x_layout=x_layout, dw_layout=dw_layout, alpha=alpha, rand_std=rand_std,
-                                algo=algo, math=math)
+                                algo=algo, math=math, topk=topk)
         self.ws = B.attach_workspace(self.desc)
 
     def logical_dw(self) -> np.ndarray:
@@ -42,6 +43,8 @@ class GpuLayer:
         d = self.dw.cpu()
         if self.dw_layout == B.DW_KRSC:
             d = I.krsc_to_kcrs(d)
+        elif self.dw_layout == B.DW_RSCK:
+            d = d.permute(3, 2, 0, 1).contiguous()
         return d.to(torch.float64).numpy()
 
     def exact(self):
@@ -53,6 +56,15 @@ class GpuLayer:
         self.dw.fill_(float("nan"))
         B.gaconv_dw_approx(method, self.x, self.dy, self.dw, self.desc, seed)
         return self.logical_dw()
+
+    def select_topk(self):
+        l = self.layer
+        t = min(self.desc.topk, l.p * l.q)
+        idx = torch.full((l.n, l.k, t), -1, dtype=torch.int32, device="cuda")
+        s = torch.full((l.n, l.k), float("nan"), dtype=torch.float32, device="cuda")
+        B.gaconv_approx_select_topk(self.dy, idx, s, self.desc)
+        torch.cuda.synchronize()
+        return idx.cpu().numpy(), s.cpu().numpy().astype(np.float64)
 
     def select(self, want_sparse=False):
         l = self.layer

@@ -21,6 +21,17 @@ def tol(dtype):
     return TOL_F32 if dtype == torch.float32 else TOL_BF16
 
 
+def top1_bound(layer, dtype):
+    """What the top-1 output must really meet, tighter than the class tolerance.  The products sum * x are formed in
+    fp32 from exactly widened inputs, and the map's sum is an fp32 tree sum (error ~1e-7 of sum|dY|), so the patch
+    accumulation meets the fp32 class whatever the input type.  Only bf16 layers with at most 64 pixels per map and
+    at least 128 input channels take the route 'sparse dY + dense tensor-core kernel', which rounds each sum to
+    bf16 once (8 significant bits, round to nearest: at most 2^-8 |sum| <= 2^-8 sum|dY| per image, i.e. 2^-8 of the
+    normaliser), plus the fp32 terms."""
+    dense = dtype == torch.bfloat16 and layer.p * layer.q <= 64 and layer.c >= 128
+    return 2.0 ** -8 + 1e-4 if dense else 1e-5
+
+
 # small cases spanning several tiles with ragged tails: C=3, W=2, stride 2, 5x5, odd sizes
 SMALL = [
     config1_layer(),
@@ -73,9 +84,11 @@ def test_top1_matches_oracle(li, dtype):
     np.put_along_axis(want, idx_ref[..., None].astype(np.int64),
                       torch.from_numpy(s).to(dtype).to(torch.float64).numpy()[..., None], axis=2)
     np.testing.assert_array_equal(sp, want)
-    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)                  # one-launch cluster kernel
+    e1 = norm_err(g.approx(B.METHOD_TOP1), ref, dn)                                  # one-launch cluster kernel, or sparse dY + dense kernel
     g2 = GpuLayer(layer, dtype, x, dy, alpha=1.0 / 128, algo=B.ALGO_DIRECT)
-    assert norm_err(g2.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)                 # select + gather kernels
+    e2 = norm_err(g2.approx(B.METHOD_TOP1), ref, dn)                                 # select + gather kernels
+    print("top-1 normalised error: auto route %.3g (bound %.3g), select+gather %.3g (bound 1e-5)" % (e1, top1_bound(layer, dtype), e2))
+    assert e1 <= top1_bound(layer, dtype) and e2 <= 1e-5
 
 
 @pytest.mark.parametrize("x_layout,dw_layout", [(B.X_NCHW, B.DW_KCRS), (B.X_NHWC, B.DW_KCRS), (B.X_NCHW, B.DW_KRSC)])
@@ -206,17 +219,19 @@ def test_schedule_run_layer_dispatches_the_scheduled_method():
 
 
 # ---- full-size layers in the configuration the benchmark times: sampled outputs + whole top-1 ----
-FULL = [("resnet", 1), ("resnet", 7), ("resnet", 13), ("resnet", 18), ("vgg", 1), ("vgg", 5), ("vgg", 9), ("vgg", 15),
-        ("cnn", 0), ("cnn", 1)]
+# (net, layer index, batch): batch 128 = the benchmark's step, batch 256 = the schedule sweep's launches
+FULL = [("resnet", 1, 128), ("resnet", 7, 128), ("resnet", 13, 128), ("resnet", 18, 128), ("vgg", 1, 128), ("vgg", 5, 128),
+        ("vgg", 9, 128), ("vgg", 15, 128), ("cnn", 0, 128), ("cnn", 1, 128),
+        ("resnet", 8, 256), ("vgg", 3, 256), ("vgg", 6, 256), ("vgg", 12, 256)]
 
 
-@pytest.mark.parametrize("net,li", FULL, ids=["%s%d" % f for f in FULL])
+@pytest.mark.parametrize("net,li,batch", FULL, ids=["%s%d_n%d" % f for f in FULL])
 @pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
-def test_full_size_layers(net, li, dtype):
-    layer = {"resnet": resnet20_layers, "vgg": vgg19_layers, "cnn": cnn2_layers}[net](128)[li]
-    if dtype == torch.float32 and net == "vgg":
-        pytest.skip("VGG-19 workload is bf16 only")
-    cfg = {"resnet": 2, "cnn": 3, "vgg": 4}[net]
+def test_full_size_layers(net, li, batch, dtype):
+    layer = {"resnet": resnet20_layers, "vgg": vgg19_layers, "cnn": cnn2_layers}[net](batch)[li]
+    if dtype == torch.float32 and (net == "vgg" or batch == 256):
+        pytest.skip("VGG-19 and the schedule sweep are bf16 workloads")
+    cfg = {"resnet": 2, "cnn": 3, "vgg": 4}[net] if batch == 128 else 5
     x, dy = I.make_layer_inputs(layer, dtype, cfg, li)
     xd, dyd = to_f64(x), to_f64(dy)
     g = GpuLayer(layer, dtype, x, dy)
@@ -227,7 +242,9 @@ def test_full_size_layers(net, li, dtype):
     np.testing.assert_array_equal(idx, idx_ref)
     assert np.max(np.abs(s - sum_ref) / abs_ref) <= TOL_SUM
     ref, dn = oracle.dw_top1(xd, dyd, sh)
-    assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
+    e1 = norm_err(g.approx(B.METHOD_TOP1), ref, dn)
+    print("top-1 normalised error %.3g (bound %.3g)" % (e1, top1_bound(layer, dtype)))
+    assert e1 <= top1_bound(layer, dtype)
     # exact: sampled output elements, each computed by the oracle on its own
     got = g.exact()
     rng = np.random.default_rng(li)
@@ -262,6 +279,9 @@ TC_SHAPES = [
     ConvLayer("tc 2x2 maps, narrow", 33, 24, 2, 2, 40, 3, 3, 1, 1),
     ConvLayer("tc 1x1 maps", 70, 32, 1, 1, 64, 1, 1, 1, 0),
     ConvLayer("tc 128->128@16 one row per CTA", 4, 128, 16, 16, 128, 3, 3, 1, 1),
+    ConvLayer("tc 512->512@4 one CTA per tile, whole output", 8, 512, 4, 4, 512, 3, 3, 1, 1),
+    ConvLayer("tc 512->512@2 one CTA per tile, whole output", 64, 512, 2, 2, 512, 3, 3, 1, 1),
+    ConvLayer("tc 256->256@8 several images per chunk, ragged batch", 21, 256, 8, 8, 256, 3, 3, 1, 1),
 ]
 
 
@@ -272,7 +292,7 @@ def test_tensor_core_exact_matches_oracle_and_direct(li):
     g = GpuLayer(layer, torch.bfloat16, x, dy, alpha=0.25, algo=B.ALGO_TENSOR)
     got = g.exact()
     assert B.gaconv_poll_async_status(g.desc) == B.OK
-    if layer.n * layer.p * layer.q * layer.k * layer.c <= 3e8:
+    if layer.n * layer.p * layer.q * layer.k * layer.c <= 4e8:
         ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.25)
         assert norm_err(got, ref, dn) <= TOL_BF16
         assert norm_err(got, ref, dn) <= 1e-4        # bf16 products are exact in fp32: far inside the class tolerance
@@ -399,3 +419,90 @@ def test_seeded_random_geometries(li):
         ref, dn = oracle.dw_top1(xd, dyd, oshape(layer))
         assert norm_err(g.approx(B.METHOD_TOP1), ref, dn) <= tol(dtype)
         assert B.gaconv_poll_async_status(g.desc) == B.OK
+
+
+# ---- inputs the paper does not discuss: NaN, infinities, signed zeros in dY (selection is still defined) ----
+def test_selection_of_nan_inf_and_signed_zero_matches_the_oracle():
+    layer = ConvLayer("specials", 2, 2, 8, 8, 6, 3, 3, 1, 1, dy_std=1.0)
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 700)
+        dy = dy.clone()
+        dy[0, 0, 3, 4] = float("inf"); dy[0, 0, 5, 1] = float("-inf")         # two infinities: the earlier
+        dy[0, 1, 2, 2] = float("inf"); dy[0, 1, 6, 6] = float("nan")           # NaN sorts above infinity
+        dy[0, 2].zero_(); dy[0, 2, 1, 1] = -0.0                                # zeros of either sign: position 0
+        dy[0, 3, 7, 7] = float("nan"); dy[0, 3, 0, 3] = float("nan")           # equal NaN payloads: the earlier
+        dy[1, 4, 4, 4] = float("-inf")
+        g = GpuLayer(layer, dtype, x, dy)
+        idx, s, _ = g.select()
+        idx_ref, sum_ref, _ = oracle.top1_select(to_f64(dy))
+        np.testing.assert_array_equal(idx, idx_ref)
+        assert idx[0, 0] == 3 * 8 + 4 and idx[0, 1] == 6 * 8 + 6 and idx[0, 2] == 0 and idx[0, 3] == 3 and idx[1, 4] == 36
+        np.testing.assert_array_equal(np.isnan(s), np.isnan(sum_ref))          # the sum propagates as IEEE does
+        np.testing.assert_array_equal(np.isinf(s), np.isinf(sum_ref))
+        g.desc.topk = 3
+        np.testing.assert_array_equal(g.select_topk()[0], oracle.topk_select(to_f64(dy), 3)[0])
+
+
+# ---- the host half of the bounded-wait report: a raised status word is reported once, then cleared ----
+def test_poll_reports_a_raised_status_word_once():
+    layer = config1_layer()
+    x, dy = _inputs(layer, torch.float32, 710)
+    g = GpuLayer(layer, torch.float32, x, dy)
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+    g.ws[:4].copy_(torch.tensor([1, 0, 0, 0], dtype=torch.uint8))              # what a kernel's give-up branch writes
+    assert B.gaconv_poll_async_status(g.desc) == B.ERR_TIMEOUT
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+    assert int(g.ws[:4].cpu().sum()) == 0
+
+
+# ---- top-k variant (Section 2.3): selection bit-exact, dW within the fp32 class for both input types ----
+TOPK_SHAPES = [
+    ConvLayer("topk 16->16@32", 4, 16, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("topk ragged s2", 3, 7, 15, 9, 5, 3, 3, 2, 0, dy_std=1.0),
+    ConvLayer("topk 4x4 c48", 6, 48, 4, 4, 40, 3, 3, 1, 1),
+    ConvLayer("topk 2x2 (k clamps to 4)", 5, 8, 2, 2, 8, 3, 3, 1, 1),
+    ConvLayer("topk 5x5", 2, 3, 16, 16, 8, 5, 5, 1, 2, x_dist="uniform_pm1"),
+]
+
+
+@pytest.mark.parametrize("topk", [1, 2, 5, 16])
+@pytest.mark.parametrize("li", range(len(TOPK_SHAPES)), ids=[l.name for l in TOPK_SHAPES])
+def test_topk_matches_oracle(li, topk):
+    layer = TOPK_SHAPES[li]
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 720 + li)
+        xd, dyd = to_f64(x), to_f64(dy)
+        g = GpuLayer(layer, dtype, x, dy, alpha=0.5, topk=topk)
+        idx, s = g.select_topk()
+        idx_ref, sum_ref, abs_ref = oracle.topk_select(dyd, topk)
+        np.testing.assert_array_equal(idx, idx_ref)
+        assert np.max(np.abs(s - sum_ref) / np.maximum(abs_ref, 1e-300)) <= TOL_SUM
+        ref, dn = oracle.dw_topk(xd, dyd, oshape(layer), topk, 0.5)
+        got = g.approx(B.METHOD_TOPK)
+        assert norm_err(got, ref, dn) <= TOL_F32
+        np.testing.assert_array_equal(got, g.approx(B.METHOD_TOPK))             # reproducible
+        if topk == 1:
+            ref1, dn1 = oracle.dw_top1(xd, dyd, oshape(layer), 0.5)
+            assert norm_err(got, ref1, dn1) <= TOL_F32
+    bad = GpuLayer(layer, torch.float32, *_inputs(layer, torch.float32, 720 + li), topk=0)
+    with pytest.raises(B.GaconvError) as e:
+        bad.approx(B.METHOD_TOPK)
+    assert e.value.status == B.ERR_BAD_DESC
+
+
+# ---- dW in the K K C_i C_o order (RSCK), through every kernel family ----
+@pytest.mark.parametrize("li", [0, 2, 5, 8, 9], ids=lambda i: SMALL[i].name)
+def test_rsck_output_layout(li):
+    layer = SMALL[li]
+    for dtype in DTYPES:
+        x, dy = _inputs(layer, dtype, 740 + li)
+        xd, dyd = to_f64(x), to_f64(dy)
+        ref, dn = oracle.dw_exact(xd, dyd, oshape(layer), 0.5)
+        ref1, dn1 = oracle.dw_top1(xd, dyd, oshape(layer), 0.5)
+        for algo in (B.ALGO_AUTO, B.ALGO_DIRECT):
+            g = GpuLayer(layer, dtype, x, dy, alpha=0.5, dw_layout=B.DW_RSCK, algo=algo)
+            assert norm_err(g.exact(), ref, dn) <= tol(dtype)
+            assert norm_err(g.approx(B.METHOD_TOP1), ref1, dn1) <= top1_bound(layer, dtype)
+        z = oracle.dw_random(ref.size, 3, 1.0 / 128).reshape(ref.shape)
+        assert np.max(np.abs(g.approx(B.METHOD_RANDOM, seed=3) - z)) <= 1e-5 * 6 / 128
+        assert np.all(g.approx(B.METHOD_ZERO) == 0)

@@ -25,10 +25,11 @@ pytestmark = pytest.mark.gpu
                          ids=["f32 direct kernel", "bf16 tensor-core kernel"])
 def test_static_scratch_entry_matches_workspace_entry_twice(dtype, layer):
     x, dy = I.make_layer_inputs(layer, dtype, 8, 0)
-    _, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer))
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer))
     tol = TOL_F32 if dtype == torch.float32 else TOL_BF16
     g = GpuLayer(layer, dtype, x, dy)
     want = g.exact()                                   # existing entry point, caller-owned workspace
+    assert norm_err(want, ref, dn) <= tol
     assert B.gaconv_workspace_size(g.desc, B.METHOD_EXACT) <= B.gaconv_static_scratch_bytes()
     # the new entry point ignores the descriptor's workspace: give it none
     bare = B.make_desc(layer, dtype)
@@ -36,7 +37,9 @@ def test_static_scratch_entry_matches_workspace_entry_twice(dtype, layer):
         g.dw.fill_(float("nan"))
         B.gaconv_dw_exact_static(g.x, g.dy, g.dw, bare)
         got = g.logical_dw()
-        assert norm_err(got, want, dn) <= tol
+        assert norm_err(got, want, dn) <= tol          # against the existing entry point
+        assert norm_err(got, ref, dn) <= tol           # and against the oracle
+        assert B.gaconv_poll_async_status_static() == B.OK
     # a different problem in between must not disturb the next one (the array keeps old contents)
     other = ConvLayer("other", 5, 8, 9, 9, 12, 3, 3, 1, 1, dy_std=1.0)
     xo, dyo = I.make_layer_inputs(other, torch.float32, 8, 1)
@@ -47,6 +50,8 @@ def test_static_scratch_entry_matches_workspace_entry_twice(dtype, layer):
     g.dw.fill_(float("nan"))
     B.gaconv_dw_exact_static(g.x, g.dy, g.dw, bare)
     assert norm_err(g.logical_dw(), want, dn) <= tol
+    assert norm_err(g.logical_dw(), ref, dn) <= tol
+    assert B.gaconv_poll_async_status_static() == B.OK
 
 
 def test_static_scratch_entry_rejects_problems_beyond_its_limit():
