@@ -1,15 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the filter-gradient (dW) hot path on B200.
 
-One "step" is one pass of the whole path over one synthetic batch of a layer set (default: the 19
-convolutions of ResNet-20 for CIFAR-10 at batch 128, inputs in bf16 and in fp32): for every layer the
-exact dW, the top-1 approximation (Algorithm 1), the zero gradient and the random gradient, each
-dispatched by the approximation-schedule driver.  The step is captured once in a CUDA graph and
-replayed; it is ordered method-major so that a buffer is touched again only after more than twice
-the L2 capacity of other data has streamed through (cold-L2 protocol).
+One "step" is one pass of the whole path over one synthetic batch of the paper's three CIFAR-10
+layer sets at batch 128 (default: VGG-19 in bf16 -- the largest single-GPU workload -- with ResNet-20
+and the two-layer CNN in bf16 and fp32 beside it): for every layer the exact dW, the top-1
+approximation (Algorithm 1), the zero gradient and the random gradient, each dispatched by the
+approximation-schedule driver.  The step is captured once in a CUDA graph and replayed; it is ordered
+method-major so that a buffer is touched again only after more than twice the L2 capacity of other
+data has streamed through (cold-L2 protocol).
 
 Prints ONE JSON line (rank 0).  `value` is microseconds per layer pass (all four methods of one
 layer in one dtype), aggregated over GPUs: step time / (layer passes per step * n_gpus).
+
+Other modes: --config 2|3|4 restricts the step to one layer set; --sweep runs the approximation-
+schedule sweep at batch 256; --layer n,c,k,hw[,r[,stride]] times one layer shape (the small,
+self-ending program the ncu captures under profiles/ are taken from).
 """
 from __future__ import annotations
 
@@ -28,7 +33,36 @@ if ROOT not in sys.path:
 
 METRIC = "dW-conv us/layer"
 UNIT = "us/layer"
-WORKLOADS = {2: "resnet20_cifar10_n128", 3: "cnn2_cifar10_n128", 4: "vgg19_cifar10_n128"}
+WORKLOADS = {0: "vgg19+resnet20+cnn2_cifar10_n128", 2: "resnet20_cifar10_n128", 3: "cnn2_cifar10_n128", 4: "vgg19_cifar10_n128"}
+ORACLE_SAMPLE_IMAGES = 2      # images per distinct layer shape that both oracle legs time (scaled to the batch)
+
+
+def workload_sets(config: int, batch: int, dtypes=None):
+    """[(config id, layers, dtype names)] of the step: config 0 = all three layer sets."""
+    from paper_1908_05460_b200.layers import layer_set
+    sets = []
+    for cfg in ((4, 2, 3) if config == 0 else (config,)):
+        names = dtypes if dtypes else (["bf16"] if cfg == 4 else ["bf16", "f32"])
+        sets.append((cfg, layer_set(cfg, batch), names))
+    return sets
+
+
+def traffic_from_profiles(kernel: str):
+    """DRAM bytes of one captured launch of `kernel`, from the table in profiles/dram_traffic.md (rows:
+    | kernel | layer | dram read B | dram write B | algorithmic B | source |).  None when no row matches."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        cells = [c.strip() for c in line.strip().strip("|").split("|")]
+        if len(cells) >= 6 and cells[0] == kernel:
+            try:
+                rd, wr, alg = int(cells[2]), int(cells[3]), int(cells[4])
+            except ValueError:
+                continue
+            return {"bytes_per_launch": rd + wr, "dram_read": rd, "dram_write": wr, "algorithmic_bytes": alg, "layer": cells[1],
+                    "source": "profiles/dram_traffic.md (" + cells[5] + "): one ncu capture, not this run"}
+    return None
 
 
 def measured_peaks():
@@ -93,7 +127,7 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------------------------
 # CPU oracle legs
-def oracle_sample_us_per_layer(layers, imgs: int):
+def oracle_sample_us_per_layer(layers, imgs: int = ORACLE_SAMPLE_IMAGES):
     """Times the oracle (exact + top-1 + zero + random) on `imgs` images of every distinct layer shape
     and extrapolates linearly in the batch size.  Returns (us per layer pass, seconds spent, threads)."""
     import numpy as np
@@ -127,21 +161,22 @@ def run_reference(args, layers):
     if rank != 0:
         return
     for _ in range(args.warmup):
-        oracle_sample_us_per_layer(layers, 1)
+        oracle_sample_us_per_layer(layers)
     vals, t0 = [], time.perf_counter()
     threads = 1
     for _ in range(args.steps):
-        v, _, threads = oracle_sample_us_per_layer(layers, 1)
+        v, _, threads = oracle_sample_us_per_layer(layers)
         vals.append(v)
     wall = time.perf_counter() - t0
     value = statistics.mean(vals)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / args.steps * 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOADS[args.config], "note": "CPU oracle; each step times 1 of 128 images per "
-                       "distinct layer shape and scales by the batch size"},
+            "config": {"workload": WORKLOADS[args.config], "note": "CPU oracle; each step times %d of %d images per "
+                       "distinct layer shape and scales by the batch size" % (ORACLE_SAMPLE_IMAGES, args.batch)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": "1 of 128 images per distinct layer shape, exact+top1+zero+random, x128"},
+                             "sample": "%d of %d images per distinct layer shape (exact+top1+zero+random, fp64), scaled to the "
+                                       "full batch" % (ORACLE_SAMPLE_IMAGES, args.batch)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -202,13 +237,65 @@ def run_sweep(args):
     print(json.dumps(out))
 
 
+def run_one_layer(args):
+    """--layer: one layer shape through the library a few times, each launch on its own copy of the inputs
+    (enough copies to exceed twice the L2 capacity unless --copies says otherwise).  Prints one line."""
+    import torch
+    from paper_1908_05460_b200 import binding as B
+    from paper_1908_05460_b200 import inputs as I
+    from paper_1908_05460_b200 import build as build_mod
+    from paper_1908_05460_b200.layers import ConvLayer
+    build_mod.build()
+    B.load()
+    v = [int(t) for t in args.layer.split(",")]
+    n, c, k, hw = v[:4]
+    r = v[4] if len(v) > 4 else 3
+    stride = v[5] if len(v) > 5 else 1
+    layer = ConvLayer("layer", n, c, hw, hw, k, r, r, stride, r // 2)
+    dname = (args.dtypes or "bf16").split(",")[0]
+    dt = torch.bfloat16 if dname == "bf16" else torch.float32
+    eb = 2 if dname == "bf16" else 4
+    x, dy = I.make_layer_inputs(layer, dt, 0, 0)
+    xg, dyg = I.to_nhwc(x).cuda(), dy.cuda()
+    nbytes = (xg.numel() + dyg.numel()) * eb
+    copies = args.copies or max(2, min(64, -(-280_000_000 // nbytes)))
+    bufs = [(xg, dyg)] + [(xg.clone(), dyg.clone()) for _ in range(copies - 1)]
+    dw = torch.empty(layer.k, layer.r, layer.s, layer.c, dtype=torch.float32, device="cuda")
+    desc = B.make_desc(layer, dt, alpha=1.0 / layer.n, topk=args.topk)
+    ws = B.attach_workspace(desc)
+    method = {"exact": B.METHOD_EXACT, "top1": B.METHOD_TOP1, "zero": B.METHOD_ZERO, "random": B.METHOD_RANDOM,
+              "topk": B.METHOD_TOPK}[args.method]
+
+    def one(xb, dyb):
+        if method == B.METHOD_EXACT:
+            B.gaconv_dw_exact(xb, dyb, dw, desc)
+        else:
+            B.gaconv_dw_approx(method, xb, dyb, dw, desc, 1)
+
+    one(*bufs[0])
+    torch.cuda.synchronize()
+    es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts = []
+    for _ in range(max(1, args.layer_iters)):
+        es.record()
+        for xb, dyb in bufs:
+            one(xb, dyb)
+        ee.record()
+        ee.synchronize()
+        ts.append(es.elapsed_time(ee) * 1e3 / copies)
+    print(json.dumps({"layer": args.layer, "dtype": dname, "method": args.method, "us_per_call_host_launched": statistics.median(ts),
+                      "copies": copies, "status": B.gaconv_poll_async_status(desc), "launches": B.gaconv_launch_count()}))
+    del ws
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4], help="layer set: 2 ResNet-20, 3 two-layer CNN, 4 VGG-19")
+    ap.add_argument("--config", type=int, default=0, choices=[0, 2, 3, 4],
+                    help="layer sets of the step: 0 all three (default), 2 ResNet-20, 3 two-layer CNN, 4 VGG-19")
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
     ap.add_argument("--layer-iters", type=int, default=5, help="per-layer timing repetitions (median)")
@@ -218,16 +305,22 @@ def main():
     ap.add_argument("--detail", default=None, help="write the per-layer table to this JSON file")
     ap.add_argument("--sweep", action="store_true", help="run the approximation-schedule sweep instead of the step benchmark")
     ap.add_argument("--sweep-batch", type=int, default=256)
+    ap.add_argument("--layer", default=None, help="n,c,k,hw[,r[,stride]]: time one layer shape and exit")
+    ap.add_argument("--method", default="exact", choices=["exact", "top1", "zero", "random", "topk"], help="method of --layer")
+    ap.add_argument("--topk", type=int, default=4, help="entries per map of --method topk")
+    ap.add_argument("--copies", type=int, default=0, help="input copies of --layer (0: enough to exceed twice the L2)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    from paper_1908_05460_b200.layers import layer_set
-    layers = layer_set(args.config, args.batch)
+    sets = workload_sets(args.config, args.batch, args.dtypes.split(",") if args.dtypes else None)
     if args.impl == "reference":
-        run_reference(args, layers)
+        run_reference(args, [l for _, ls, _ in sets for l in ls])
         return
     if args.sweep:
         run_sweep(args)
+        return
+    if args.layer:
+        run_one_layer(args)
         return
 
     import torch
@@ -246,31 +339,33 @@ def main():
         dist.barrier()
     B.load()
     peaks = measured_peaks()
-
-    dtype_names = (args.dtypes.split(",") if args.dtypes else (["bf16"] if args.config == 4 else ["bf16", "f32"]))
-    dtypes = [{"bf16": torch.bfloat16, "f32": torch.float32}[d] for d in dtype_names]
+    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}
 
     # ---- inputs: generated on the host (seeded), resident in HBM before any timed region ----
     class Slot:
         pass
     slots = []
     h2d = d2h = 0
-    for dt, dname in zip(dtypes, dtype_names):
-        for li, l in enumerate(layers):
-            s = Slot()
-            s.layer, s.li, s.dtype, s.dname = l, li, dt, dname
-            x, dy = I.make_layer_inputs(l, dt, args.config, li + 1000 * rank)
-            s.x_host = I.to_nhwc(x).pin_memory(); s.dy_host = dy.contiguous().pin_memory()
-            s.x = s.x_host.cuda(); s.dy = s.dy_host.cuda()
-            s.dw = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32, device="cuda")
-            s.dw_host = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32).pin_memory()
-            s.desc = B.make_desc(l, dt, alpha=1.0 / l.n)
-            s.ws = B.attach_workspace(s.desc)
-            s.eb = 2 if dt == torch.bfloat16 else 4
-            h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs
-            d2h += 4 * s.dw.numel() * 4
-            slots.append(s)
-    L = len(layers)
+    for cfg, layers, dtype_names in sets:
+        for dname in dtype_names:
+            for li, l in enumerate(layers):
+                s = Slot()
+                s.layer, s.li, s.dtype, s.dname, s.cfg = l, len([t for t in slots if t.cfg == cfg and t.dname == dname]), tdt[dname], dname, cfg
+                s.net = {2: "resnet20", 3: "cnn2", 4: "vgg19"}[cfg]
+                x, dy = I.make_layer_inputs(l, s.dtype, cfg, li + 1000 * rank)
+                s.x_host = I.to_nhwc(x).pin_memory(); s.dy_host = dy.contiguous().pin_memory()
+                s.x = s.x_host.cuda(); s.dy = s.dy_host.cuda()
+                s.dw = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32, device="cuda")
+                s.dw_host = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32).pin_memory()
+                s.desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n)
+                s.ws = B.attach_workspace(s.desc)
+                s.eb = 2 if s.dtype == torch.bfloat16 else 4
+                h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs
+                d2h += 4 * s.dw.numel() * 4
+                slots.append(s)
+    L = len(slots)
+    for i, s in enumerate(slots):
+        s.sid = i                      # layer index within the step's schedule
     input_bytes = sum((s.x.numel() + s.dy.numel()) * s.eb for s in slots)
 
     methods = [("exact", B.METHOD_EXACT), ("top1", B.METHOD_TOP1), ("zero", B.METHOD_ZERO), ("random", B.METHOD_RANDOM)]
@@ -279,7 +374,7 @@ def main():
               for _, m in methods}
 
     def run_one(s, m, t):
-        scheds[m].run_layer(s.li, 4 * t + (3 if m >= 0 else 0), s.x, s.dy, s.dw, s.desc)
+        scheds[m].run_layer(s.sid, 4 * t + (3 if m >= 0 else 0), s.x, s.dy, s.dw, s.desc)
 
     def step(t):
         for _, m in methods:                # method-major: a buffer is reused only after a full input pass
@@ -354,7 +449,7 @@ def main():
 
         def burst():
             for xb, dyb in bufs:
-                scheds[m].run_layer(s.li, step_no, xb, dyb, s.dw, s.desc)
+                scheds[m].run_layer(s.sid, step_no, xb, dyb, s.dw, s.desc)
         burst()
         torch.cuda.synchronize()
         gr = torch.cuda.CUDAGraph()
@@ -371,14 +466,19 @@ def main():
         return statistics.median(ts)
 
     empty_pair_us = isolated_us(lambda: None, 20)
-    table = []
+    table, seen = [], {}
     for s in (slots if args.layer_iters > 0 else []):
-        row = {"layer": s.layer.name, "index": s.li, "dtype": s.dname}
-        for name, m in methods:
-            row[name + "_us"] = streamed_us(s, m, args.layer_iters)
-        for name, m in methods[:2]:
-            row[name + "_isolated_us"] = isolated_us(lambda: run_one(s, m, 2), 5)
         l = s.layer
+        key = (s.dname, l.c, l.k, l.h, l.r, l.stride)       # layers of one shape share one measurement
+        if key not in seen:
+            row = {}
+            for name, m in methods:
+                row[name + "_us"] = streamed_us(s, m, args.layer_iters)
+            for name, m in methods[:2]:
+                row[name + "_isolated_us"] = isolated_us(lambda: run_one(s, m, 2), 5)
+            seen[key] = row
+        row = dict(seen[key])
+        row.update({"layer": l.name, "net": s.net, "index": s.li, "dtype": s.dname})
         fl, be, bt = l.flops_exact(), l.bytes_exact(s.eb), l.bytes_top1(s.eb)
         t_tensor = fl / (peaks["bf16_tflops"] * 1e12 * (1.0 if s.eb == 2 else 0.5)) * 1e6   # tf32 nominal ratio 1/2
         t_hbm = be / (peaks["hbm_gbs"] * 1e9) * 1e6
@@ -391,30 +491,31 @@ def main():
         table.append(row)
     sum_us = {name: sum(r[name + "_us"] for r in table) for name, _ in methods}
 
-    # ---- roofline of the dominant kernel family (largest share of the per-layer time) ----
-    fam = max(("exact", "top1"), key=lambda n: sum_us[n])
-    if not table:
-        roof = {"bound": None, "achieved": None, "peak": None, "unit": None, "kernel": None, "launches": 0}
-    elif fam == "exact":
-        hb = [r for r in table if r["exact_bound"] == "hbm"]; tb = [r for r in table if r["exact_bound"] == "tensor"]
-        if sum(r["exact_us"] for r in hb) >= sum(r["exact_us"] for r in tb):
-            ach = sum(r["exact_bytes"] for r in hb) / sum(r["exact_us"] for r in hb) / 1e3
-            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "kernel": "exact dW",
-                    "launches": len(hb)}
-        else:
-            ach = sum(r["gflop"] for r in tb) / sum(r["exact_us"] for r in tb) * 1e3   # GFLOP/us -> TFLOP/s
-            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "kernel": "exact dW", "launches": len(tb)}
-    else:
-        ach = sum(r["top1_bytes"] for r in table) / sum_us["top1"] / 1e3
-        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "kernel": "top-1 select+gather", "launches": len(table)}
-    roof["frac"] = roof["achieved"] / roof["peak"] if table else None
-    roof["peak_source"] = peaks["source"]
-    # DRAM bytes of one launch from the committed ncu capture of this kernel family (profiles/): the exact
-    # fp32 kernel on 16->16@32x32, N=128 moved 16.80 MB for 16.79 MB of algorithmic bytes (no re-reads)
-    roof["traffic"] = {"bytes_per_launch": 16800768, "algorithmic_bytes": 16786432, "layer": "16->16@32 f32 N=128",
-                       "source": "profiles/direct_mma_f32_16x16_32x32_n128.md"} if roof.get("kernel") == "exact dW" else None
+    # ---- roofline per kernel family: exact dW on tensor-bound layers, exact dW on HBM-bound layers, top-1 ----
+    # a family's fraction = sum of the layers' roofline times / sum of their measured times
+    roof = {"bound": None, "achieved": None, "peak": None, "unit": None, "kernel": None, "frac": None, "traffic": None}
+    if table:
+        tb = [r for r in table if r["exact_bound"] == "tensor"]; hb = [r for r in table if r["exact_bound"] == "hbm"]
+        fams = {}
+        if tb:
+            t = sum(r["exact_us"] for r in tb)
+            # fp32 layers count at the TF32 peak (half the bf16 peak): FLOPs scaled to bf16-equivalents
+            eq = sum(r["gflop"] * (1.0 if r["dtype"] == "bf16" else 2.0) for r in tb)
+            fams["exact_tensor_bound"] = {"bound": "tensor", "achieved": eq / t * 1e3, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                          "frac": sum(r["exact_roof_us"] for r in tb) / t, "layers": len(tb), "sum_us": t,
+                                          "note": "bf16-equivalent TFLOP/s (fp32 layers counted at the TF32 peak, half the bf16 peak)"}
+        if hb:
+            t = sum(r["exact_us"] for r in hb)
+            fams["exact_hbm_bound"] = {"bound": "hbm", "achieved": sum(r["exact_bytes"] for r in hb) / t / 1e3, "peak": peaks["hbm_gbs"],
+                                       "unit": "GB/s", "frac": sum(r["exact_roof_us"] for r in hb) / t, "layers": len(hb), "sum_us": t}
+        t = sum_us["top1"]
+        fams["top1"] = {"bound": "hbm", "achieved": sum(r["top1_bytes"] for r in table) / t / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": sum(r["top1_bytes"] for r in table) / (peaks["hbm_gbs"] * 1e3) / t, "layers": len(table), "sum_us": t}
+        dom = max(fams, key=lambda f: fams[f]["sum_us"])
+        kernel = {"exact_tensor_bound": "exact_tc_kernel", "exact_hbm_bound": "exact_tc_kernel", "top1": "top1_fused_kernel"}[dom]
+        roof = {k: fams[dom][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
+        roof.update({"kernel": kernel, "family": dom, "peak_source": peaks["source"], "families": fams,
+                     "traffic": traffic_from_profiles(kernel)})
 
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
     e2e = None
@@ -426,7 +527,6 @@ def main():
         e2e_step(0)
         barrier()
         k2 = max(1, min(args.steps, 3))
-        t0 = time.perf_counter()
         ev0.record()
         for t in range(k2):
             e2e_step(t)
@@ -443,21 +543,23 @@ def main():
 
     cpu = None
     if not args.no_cpu:
-        imgs, spent = 1, 0.0
-        v, spent, threads = oracle_sample_us_per_layer(layers, imgs)
-        while spent < 6.0 and imgs < args.batch:
-            imgs *= 4
-            v, spent, threads = oracle_sample_us_per_layer(layers, imgs)
+        v, spent, threads = oracle_sample_us_per_layer([s.layer for s in slots])
         cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": "%d of %d images per distinct layer shape (exact+top1+zero+random, fp64), scaled to the "
-                         "full batch; %.1f s of CPU work" % (min(imgs, args.batch), args.batch, spent)}
+                         "full batch; %.1f s of CPU work" % (ORACLE_SAMPLE_IMAGES, args.batch, spent)}
 
+    nets = {}
+    for r in table:
+        d = nets.setdefault(r["net"] + "/" + r["dtype"], {"layers": 0, "exact_us": 0.0, "top1_us": 0.0, "exact_roof_us": 0.0})
+        d["layers"] += 1; d["exact_us"] += r["exact_us"]; d["top1_us"] += r["top1_us"]; d["exact_roof_us"] += r["exact_roof_us"]
+    dnames = sorted({s.dname for s in slots})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "+".join(dtype_names) + " inputs, f32 accumulate", "data": "synthetic",
-        "config": {"workload": "%s (%d conv layers x {%s} x {exact, top1, zero, random})"
-                               % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), L, ",".join(dtype_names)),
+        "dtype": "+".join(dnames) + " inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "%s (%d layer passes x {exact, top1, zero, random}; sets: %s)"
+                               % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), passes,
+                                  ", ".join("%s %s" % ({2: "resnet20", 3: "cnn2", 4: "vgg19"}[c], "/".join(dn)) for c, _, dn in sets)),
                    "layer_passes_per_step": passes, "cuda_graph": graph is not None,
                    "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
                          "order); per-layer timings stream over rotating input copies > 2.5x L2" % (input_bytes / 1e6)},
@@ -465,7 +567,8 @@ def main():
         "roofline": roof, "cpu_baseline": cpu,
         "breakdown_us": {"streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
                          "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
-                         "top1_speedup_over_exact": (sum_us["exact"] / sum_us["top1"]) if table else None},
+                         "top1_speedup_over_exact": (sum_us["exact"] / sum_us["top1"]) if table else None,
+                         "per_set": nets},
         "paper_context": "paper reports >7% training wall-clock speedup (ResNet-20/VGG-19, Titan Xp, TF 1.13, cuDNN 7.4.2)",
     }
     if args.detail:

@@ -27,7 +27,23 @@ def headers() -> list[str]:
         + glob.glob(os.path.join(ROOT, "include", "*.h"))
 
 
+def _flags(verbose: bool = False) -> list[str]:
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
+             "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    if os.environ.get("GACONV_TUNING", "") not in ("", "0"):
+        flags.append("-DGACONV_TUNING")
+    if verbose:
+        flags.append("-Xptxas=-v")
+    return flags
+
+
+def _flags_tag() -> str:
+    return os.path.join(OBJ, "flags.txt")
+
+
 def stale() -> bool:
+    """True when the library is missing or older than a source or header.  (Which variant the existing library is
+    -- default or tuning -- is not checked here: a library shipped to a machine is used as it is.)"""
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
@@ -35,19 +51,14 @@ def stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not stale():
+    flags = _flags(verbose)
+    tag = _flags_tag()
+    same_flags = os.path.exists(tag) and open(tag).read() == " ".join(flags)
+    explicit_variant = "GACONV_TUNING" in os.environ          # the caller asked for a variant: rebuild if it differs
+    if not force and not stale() and (same_flags or not explicit_variant):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tuning = os.environ.get("GACONV_TUNING", "") not in ("", "0")
-    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
-             "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-    if tuning:
-        flags.append("-DGACONV_TUNING")
-    if verbose:
-        flags.append("-Xptxas=-v")
     os.makedirs(OBJ, exist_ok=True)
-    tag = os.path.join(OBJ, "flags.txt")
-    same_flags = os.path.exists(tag) and open(tag).read() == " ".join(flags)
     hdr_time = max(os.path.getmtime(h) for h in headers())
 
     def compile_one(src: str) -> str:

@@ -101,6 +101,12 @@ struct TcParams {
     int b_tiles;        // S (halo) or R*S; 1 when wide
     int tiny;           // 1: maps of fewer than 64 pixels: A comes from a transposed copy dYt[n][pq][k] (MN-major,
                         //    64 channels per 128-byte row); chunks are whole images, 16 reduction rows per k-step
+    int tiny2;          // with tiny, for single-row CTAs of stride-1 layers: the reduction rows of a chunk of ci (8, 16 or 32) images
+                        //    are ordered (pixel, image).  Then ONE X tile with a column halo, laid out [row][column][image][channel]
+                        //    by a tensor map with permuted dimensions, serves all column shifts (a shift = one pixel = ci 128-byte
+                        //    rows), as the wide tile does for maps of 64 pixels and more
+    int b_lbo;          // B descriptor: bytes between the column-shift atoms of an MMA
+    int b_sub_bytes;    // B descriptor advance from one A box (or image row) to the next
     int by_image;       // 1: a chunk is ci whole images (maps under 64 pixels)
     int a_k4_step;      // descriptor advance (16-byte units) from one k-step to the next inside an A box
     int a_lbo;          // leading byte offset of the A descriptor
@@ -219,7 +225,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             const uint32_t sb = sa + P.a_region_bytes;
             for (int b = lane; b < n_all; b += 32) {
                 if (b < n_a) {
-                    if (P.tiny) {                                                // one box per 64-channel atom
+                    if (P.tiny2) {                                               // one box per 64-channel atom, [pixel][image][k]
+                        tma_load_3d(sa + b * P.a_lbo, &map_dy, full, k0 + 64 * b, n0, 0);
+                    } else if (P.tiny) {                                         // one box per 64-channel atom, [image][pixel][k]
                         tma_load_3d(sa + b * P.a_lbo, &map_dy, full, k0 + 64 * b, 0, n0);
                     } else if (P.by_image) {
                         tma_load_3d(sa, &map_dy, full, 0, k0, n0);               // ci whole maps in one box
@@ -229,7 +237,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                     }
                 } else {
                     const int j = b - n_a;
-                    if (P.wide) {
+                    if (P.tiny2) {                                               // dimensions (c, n, w, h)
+                        tma_load_4d(sb, &map_x, full, c0, n0, -g.pad_w, r_lo - g.pad_h);
+                    } else if (P.wide) {
                         tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
                     } else if (P.halo) {
                         tma_load_4d(sb + j * P.b_tile_stride, &map_x, full, c0, j - g.pad_w, p0 - g.pad_h, n0);
@@ -257,7 +267,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         // stride between the two 8-pixel halves of a k-step: contiguous, except in wide mode when a k-step spans two rows
         const uint32_t b_sbo = (P.wide && g.q == 8) ? wt * b_row_bytes : 8 * b_row_bytes;
         const uint32_t b_hi = (b_sbo >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
-        const uint32_t a_lo_c = (((uint32_t)P.a_lbo >> 4) & 0x3fffu) << 16, b_lo_c = (((P.wide ? b_row_bytes : (uint32_t)P.b_tile_stride) >> 4) & 0x3fffu) << 16;
+        const uint32_t a_lo_c = (((uint32_t)P.a_lbo >> 4) & 0x3fffu) << 16, b_lo_c = (((uint32_t)P.b_lbo >> 4) & 0x3fffu) << 16;
         const int ks_per_sub = P.a_sub_px / 16;
         const uint32_t a_k4 = (uint32_t)P.a_k4_step;
         const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4;
@@ -267,7 +277,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4)
             b_k_off[k4] = (P.wide ? (((16u * k4) / g.q) * wt + (16u * k4) % g.q) * b_row_bytes : 16u * k4 * b_row_bytes) >> 4;
-        const uint32_t b_sub_step = (P.wide ? (uint32_t)(P.a_sub_px / g.q) * wt * b_row_bytes : (uint32_t)P.a_sub_px * b_row_bytes) >> 4;
+        const uint32_t b_sub_step = (uint32_t)P.b_sub_bytes >> 4;
         const int R = R_T ? R_T : P.rc;
         const int KS = KS_T ? KS_T : ks_per_sub;
         // this issuer's filter rows: TMEM address of the accumulator and descriptor offset of the row
@@ -671,7 +681,10 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.b_swz = swz_code(ct * 2);
     // wide tile: stride 1, whole rows per chunk, k-steps inside a row (Q a multiple of 16) or exactly two rows (Q = 8)
     P.wide = (env_int("GACONV_TC_WIDE", 1) && !small_map && g.stride_h == 1 && (g.q % 16 == 0 || g.q == 8) && 64 % g.q == 0) ? 1 : 0;
-    P.b_tiles = P.wide ? 1 : halo ? g.s : P.rc * g.s;
+    // small maps, one filter row per CTA: the (pixel, image) ordering with a single haloed X tile
+    const bool tiny2 = tiny && P.rc == 1 && g.stride_h == 1 && g.q % 2 == 0 && g.n >= 8 && env_int("GACONV_TC_TINY2", 1);
+    P.tiny2 = tiny2 ? 1 : 0;
+    P.b_tiles = (P.wide || tiny2) ? 1 : halo ? g.s : P.rc * g.s;
 
     // chunk size: as many rows (or images) as fit the stage budget.  The hand-over of a stage costs the producer
     // and the issuer several hundred cycles each, so a stage should carry at least ~8 MMAs.
@@ -686,7 +699,13 @@ bool plan_tc(const Geom& g, TcPlan* out)
         return a_bytes + P.b_tiles * *tile_stride;
     };
     int ci = 1, bp = small_map ? g.p : 64 / g.q, a_subs, tb, ts;
-    if (tiny) {
+    auto tiny2_stage = [&](int c) { return ((P.m / 64) * c * pq * 128 + 1023) / 1024 * 1024 + (g.p * (g.q + g.s - 1) * c * 128 + 1023) / 1024 * 1024; };
+    if (tiny2) {
+        // reduction rows ordered (pixel, image): a k-step = 16 rows = two pixels x 8 images, one pixel x 16, or half a pixel's 32;
+        // as many images per chunk as keep an image row within four k-steps and the stage within the budget
+        ci = 8;
+        while (ci * 2 <= 32 && g.q * ci * 2 / 16 <= 4 && ci * 2 <= g.n && tiny2_stage(ci * 2) <= budget) ci *= 2;
+    } else if (tiny) {
         ci = 64 / pq;                                   // 64 reduction rows = four k-steps per chunk at least
         while (ci * 2 * pq <= 256 && ci * 2 <= g.n && stage_bytes(ci * 2, bp, &a_subs, &tb, &ts) <= budget) ci *= 2;
     } else if (small_map) {
@@ -702,10 +721,19 @@ bool plan_tc(const Geom& g, TcPlan* out)
     }
     P.ci = ci; P.bp = bp;
     P.stage_bytes = stage_bytes(ci, bp, &a_subs, &tb, &ts);
+    if (tiny2) {                                        // A: [pixel][image][64 k] per atom; B: [row][column + halo][image][64 c]
+        a_subs = g.p;                                   // the issuer walks image rows: Q pixels x ci images = Q * ci / 16 k-steps each
+        P.a_sub_px = ci * g.q;
+        tb = g.p * (g.q + g.s - 1) * ci * 128;
+        ts = (tb + 1023) / 1024 * 1024;
+        P.stage_bytes = tiny2_stage(ci);
+    }
     P.stage_bytes = (P.stage_bytes + 1023) / 1024 * 1024;
     P.a_subs = a_subs; P.b_tile_bytes = tb; P.b_tile_stride = ts;
     P.a_subs_img = (tiny || small_map) ? a_subs : a_subs / ci;
-    P.a_sub_bytes = tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
+    P.a_sub_bytes = tiny2 ? ci * g.q * 128 : tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
+    P.b_lbo = tiny2 ? ci * 128 : P.wide ? ct * 2 : ts;
+    P.b_sub_bytes = tiny2 ? (g.q + g.s - 1) * ci * 128 : P.wide ? (P.a_sub_px / g.q) * (g.q + g.s - 1) * ct * 2 : P.a_sub_px * ct * 2;
     P.a_k4_step = tiny ? (16 * 128) >> 4 : 2;
     P.a_lbo = tiny ? ci * pq * 128 : 16;               // tiny: bytes between the 64-channel atoms of an A tile
     P.a_region_bytes = ((tiny ? (P.m / 64) * ci * pq * 128 : P.a_subs * P.a_sub_bytes) + 1023) / 1024 * 1024;
@@ -763,8 +791,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.timeline = env_int("GACONV_TC_TIMELINE", 0);
 #ifdef GACONV_TUNING
     if (env_int("GACONV_TC_VERBOSE", 0))
-        fprintf(stderr, "plan_tc c%d k%d pq%d: m%d ct%d rsplit%d dual%d wide%d tiny%d ci%d bp%d ksteps%d stage %d B x%d, tiles %d splits %d cl %d chunks %d\n",
-                g.c, g.k, pq, P.m, ct, P.rsplit, P.dual, P.wide, P.tiny, ci, bp, P.ksteps, P.stage_bytes, P.stages, tiles, splits, cl, P.chunks);
+        fprintf(stderr, "plan_tc c%d k%d pq%d: m%d ct%d rsplit%d dual%d wide%d tiny%d/%d ci%d bp%d ksteps%d stage %d B x%d, tiles %d splits %d cl %d chunks %d\n",
+                g.c, g.k, pq, P.m, ct, P.rsplit, P.dual, P.wide, P.tiny, P.tiny2, ci, bp, P.ksteps, P.stage_bytes, P.stages, tiles, splits, cl, P.chunks);
 #endif
 
     out->partial_bytes = splits / cl > 1 ? (size_t)tiles * (splits / cl) * P.slot_quads * 16 : 0;
@@ -785,7 +813,7 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     if (enc == nullptr) return cudaErrorNotSupported;
 
     CUtensorMap map_dy, map_x;
-    if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) with 64-channel boxes
+    if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) -- (k, n, pq) for the (pixel, image) ordering -- with 64-channel boxes
         if (launch_kernel(transpose_dy_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
                           static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.k, pq) != cudaSuccess)
             return cudaErrorLaunchFailure;
@@ -794,6 +822,11 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
         cuuint64_t strides[2] = {(cuuint64_t)g.k * 2, (cuuint64_t)g.k * pq * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)pq, (cuuint32_t)P.ci};
         cuuint32_t es[3] = {1, 1, 1};
+        if (P.tiny2) {      // the same array seen as (k, n, pq): a box lands as [pixel][image][k]
+            dims[1] = (cuuint64_t)g.n; dims[2] = (cuuint64_t)pq;
+            strides[0] = (cuuint64_t)g.k * pq * 2; strides[1] = (cuuint64_t)g.k * 2;
+            box[1] = (cuuint32_t)P.ci; box[2] = (cuuint32_t)pq;
+        }
         if (enc(&map_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, scratch, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
@@ -813,6 +846,12 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
         const int cols = P.wide ? g.q + g.s - 1 : g.q * g.stride_w;
         cuuint32_t box[4] = {(cuuint32_t)P.ct, (cuuint32_t)cols, (cuuint32_t)(rows * g.stride_h), (cuuint32_t)P.ci};
         cuuint32_t es[4] = {1, (cuuint32_t)g.stride_w, (cuuint32_t)g.stride_h, 1};
+        if (P.tiny2) {      // X seen as (c, n, w, h): a box of P rows x (Q + S - 1) columns x ci images lands as [row][column][image][c]
+            dims[1] = (cuuint64_t)g.n; dims[2] = (cuuint64_t)g.w; dims[3] = (cuuint64_t)g.h;
+            strides[0] = (cuuint64_t)g.h * g.w * g.c * 2; strides[1] = (cuuint64_t)g.c * 2; strides[2] = (cuuint64_t)g.w * g.c * 2;
+            box[1] = (cuuint32_t)P.ci; box[2] = (cuuint32_t)(g.q + g.s - 1); box[3] = (cuuint32_t)g.p;
+            es[1] = es[2] = es[3] = 1;
+        }
         if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(P.ct * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -845,6 +884,8 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     GACONV_TC_CASE(3, 1)
     GACONV_TC_CASE(5, 4)
     GACONV_TC_CASE(1, 4)
+    GACONV_TC_CASE(1, 2)
+    GACONV_TC_CASE(1, 1)
     GACONV_TC_CASE(0, 0)
 #undef GACONV_TC_CASE
     if (err != cudaSuccess) return err;
