@@ -268,7 +268,10 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     float* sum = reinterpret_cast<float*>(ws + L.sum_off);
     if (L.dense && desc->algo != GACONV_ALGO_DIRECT) {
         void* sparse = ws + L.sparse_off;
-        if (launch_select(dy, idx, sum, sparse, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        if (L.tp.reads_transposed_dy) {       // the dense kernel's operand layout is written directly: no separate transpose
+            if (launch_select_sparse_transposed(dy, ws + L.scratch_off, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+            sparse = nullptr;
+        } else if (launch_select(dy, idx, sum, sparse, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
         return launch_tc(x, sparse, dw, reinterpret_cast<float*>(ws + L.partial_off), ws + L.scratch_off,
                          reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), L.tp,
                          cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;

@@ -71,6 +71,9 @@ cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int spl
 cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_sparse, const Geom& g,
                           cudaStream_t stream);
 
+// selection written as the transposed sparse tensor dYt'[n][j][k] (bf16, maps of fewer than 64 pixels, k % 8 == 0)
+cudaError_t launch_select_sparse_transposed(const void* dy, void* dyt, const Geom& g, cudaStream_t stream);
+
 // ---- gather-accumulate (Algorithm 1, patch accumulation line) ----
 struct GatherPlan {
     int chunks;          // CTAs per output channel, each owning a contiguous range of images
@@ -124,9 +127,11 @@ cudaError_t launch_stem(const void* x, const void* dy, float* dw, float* partial
 struct TcPlan {
     size_t partial_bytes;
     size_t scratch_bytes;                   // extra device scratch (transposed dY for very small maps)
+    bool reads_transposed_dy;               // the kernel's dY operand is the transposed copy dYt[n][pq][k] in the scratch
     alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
 };
 bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel
+// dy == nullptr: the scratch already holds the transposed operand (plan.reads_transposed_dy only)
 cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* counters,
                       uint32_t* status,
                       const TcPlan& plan, cudaStream_t stream);

@@ -797,6 +797,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
 
     out->partial_bytes = splits / cl > 1 ? (size_t)tiles * (splits / cl) * P.slot_quads * 16 : 0;
     out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
+    out->reads_transposed_dy = tiny;
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
     memcpy(out->opaque, &P, sizeof(P));
     return encode_fn() != nullptr;
@@ -814,10 +815,12 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
 
     CUtensorMap map_dy, map_x;
     if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) -- (k, n, pq) for the (pixel, image) ordering -- with 64-channel boxes
-        if (launch_kernel(transpose_dy_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
-                          static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.k, pq) != cudaSuccess)
-            return cudaErrorLaunchFailure;
-        note_launch();
+        if (dy != nullptr) {
+            if (launch_kernel(transpose_dy_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
+                              static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.k, pq) != cudaSuccess)
+                return cudaErrorLaunchFailure;
+            note_launch();
+        }
         cuuint64_t dims[3] = {(cuuint64_t)g.k, (cuuint64_t)pq, (cuuint64_t)g.n};
         cuuint64_t strides[2] = {(cuuint64_t)g.k * 2, (cuuint64_t)g.k * pq * 2};
         cuuint32_t box[3] = {64, (cuuint32_t)pq, (cuuint32_t)P.ci};

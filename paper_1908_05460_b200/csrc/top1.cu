@@ -149,6 +149,41 @@ select_kernel(const T* __restrict__ dy, int32_t* __restrict__ idx, float* __rest
     }
 }
 
+// Selection for the route "sparse dY + dense tensor-core kernel" on maps of fewer than 64 pixels, where that kernel
+// reads a transposed copy dYt[n][j][k] of its dY operand: writes the sparse tensor straight in that layout (the
+// signed sum, rounded to bf16, at the retained position of every map, zero elsewhere).  A block takes 64 channels
+// of one image: one thread per map scans its pq <= 32 elements, then the block writes pq rows of up to 128 bytes.
+__global__ void __launch_bounds__(128)
+select_sparse_transposed_kernel(const __nv_bfloat16* __restrict__ dy, __nv_bfloat16* __restrict__ dyt, int k, int pq)
+{
+    __shared__ int s_idx[64];
+    __shared__ unsigned short s_val[64];
+    pdl_release_next_grid();
+    const int kgroups = (k + 63) / 64;
+    const int n = blockIdx.x / kgroups, k0 = (blockIdx.x - n * kgroups) * 64, kg = min(64, k - k0);
+    pdl_wait_prior_grid();
+    if ((int)threadIdx.x < kg) {
+        const __nv_bfloat16* map = dy + ((size_t)n * k + k0 + threadIdx.x) * pq;
+        Scan sc{-1, 0, 0.0f};
+        for (int j = 0; j < pq; ++j) Elem<__nv_bfloat16>::visit1(map, j, sc);
+        s_idx[threadIdx.x] = sc.best_j;
+        s_val[threadIdx.x] = __bfloat16_as_ushort(__float2bfloat16_rn(sc.sum));
+    }
+    __syncthreads();
+    const int k8 = kg >> 3;
+    for (int item = threadIdx.x; item < pq * k8; item += blockDim.x) {
+        const int j = item / k8, q = item - j * k8;
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t lo = s_idx[8 * q + 2 * i] == j ? s_val[8 * q + 2 * i] : 0u;
+            const uint32_t hi = s_idx[8 * q + 2 * i + 1] == j ? s_val[8 * q + 2 * i + 1] : 0u;
+            w[i] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(dyt + ((size_t)n * pq + j) * k + k0 + 8 * q) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 // Selection of the top-k variant: one warp per map.  Round t picks the largest key below the key picked in
 // round t-1, where key = (bit pattern of |v|, complement of the position): keys are distinct, larger magnitude
 // first and, among equal magnitudes, the lower position first -- the order the single arg-max uses.
@@ -422,6 +457,14 @@ cudaError_t launch_select(const void* dy, int32_t* idx, float* sum, void* dy_spa
     }
     note_launch();
     return cudaGetLastError();
+}
+
+cudaError_t launch_select_sparse_transposed(const void* dy, void* dyt, const Geom& g, cudaStream_t stream)
+{
+    cudaError_t e = launch_kernel(select_sparse_transposed_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
+                                  static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(dyt), g.k, g.p * g.q);
+    note_launch();
+    return e;
 }
 
 cudaError_t launch_select_topk(const void* dy, int32_t* idx, float* sum, const Geom& g, int topk, cudaStream_t stream)
