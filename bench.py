@@ -195,7 +195,7 @@ def run_sweep(args):
     build_mod.build()
     B.load()
     torch.cuda.set_device(0)
-    out = {"workload": "schedule sweep, N=%d, bf16, seeded mask on odd steps, top-1 method" % args.sweep_batch, "nets": {}}
+    out = {"workload": "schedule sweep, N=%d, bf16, seeded mask on odd steps, top-1 method, %d lanes" % (args.sweep_batch, args.lanes), "nets": {}}
     es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for cfg, name in ((2, "resnet20"), (4, "vgg19")):
         layers = layer_set(cfg, args.sweep_batch)
@@ -210,10 +210,10 @@ def run_sweep(args):
         for f in (0.0, 0.25, 0.5, 0.75, 1.0):
             sched = B.Schedule(L, B.SCHED_SEEDED_FRACTION_ALT_BATCH, B.METHOD_TOP1, f, 20260101)
             graphs = {}
+            packed = sched.pack_step([sl[0] for sl in slots], [sl[1] for sl in slots], [sl[2] for sl in slots], [sl[3] for sl in slots])
             for parity in (0, 1):                       # one CUDA graph per step parity: the switch costs nothing
                 def one_step(t=parity):
-                    for li, (x, dy, dw, d, _) in enumerate(slots):
-                        sched.run_layer(li, t, x, dy, dw, d)
+                    sched.run_step(t, packed, lanes=args.lanes)
                 one_step(); torch.cuda.synchronize()
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
@@ -299,6 +299,7 @@ def main():
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
     ap.add_argument("--layer-iters", type=int, default=5, help="per-layer timing repetitions (median)")
+    ap.add_argument("--lanes", type=int, default=4, help="streams on which the layers of a step run next to one another (1..8)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -376,10 +377,12 @@ def main():
     def run_one(s, m, t):
         scheds[m].run_layer(s.sid, 4 * t + (3 if m >= 0 else 0), s.x, s.dy, s.dw, s.desc)
 
+    packed = {m: scheds[m].pack_step([s.x for s in slots], [s.dy for s in slots], [s.dw for s in slots], [s.desc for s in slots])
+              for _, m in methods}
+
     def step(t):
         for _, m in methods:                # method-major: a buffer is reused only after a full input pass
-            for s in slots:
-                run_one(s, m, t)
+            scheds[m].run_step(4 * t + (3 if m >= 0 else 0), packed[m], lanes=args.lanes)
 
     def barrier():
         if world > 1:
@@ -560,7 +563,7 @@ def main():
         "config": {"workload": "%s (%d layer passes x {exact, top1, zero, random}; sets: %s)"
                                % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), passes,
                                   ", ".join("%s %s" % ({2: "resnet20", 3: "cnn2", 4: "vgg19"}[c], "/".join(dn)) for c, _, dn in sets)),
-                   "layer_passes_per_step": passes, "cuda_graph": graph is not None,
+                   "layer_passes_per_step": passes, "cuda_graph": graph is not None, "lanes": args.lanes,
                    "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
                          "order); per-layer timings stream over rotating input copies > 2.5x L2" % (input_bytes / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,

@@ -193,6 +193,19 @@ int32_t gaconv_schedule_method(const gaconv_schedule_t *sched, int32_t layer, in
 gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t *sched, int32_t layer, int64_t step,
                                           const void *x, const void *dy, float *dw,
                                           const gaconv_conv_desc_t *desc, void *stream);
+/* One training step (Sections 2.5 and 3: at every batch the schedule picks, layer by layer, the exact or an
+ * approximated filter gradient): gaconv_schedule_run_layer for layers 0..num_layers-1, layer l on lane
+ * l % lanes.  Lane 0 is `stream`; the other lanes are streams the library owns (created on first use, one set
+ * per device), forked from `stream` when the call starts and joined back into it before it returns, so for the
+ * caller the whole step is ordered like one operation on `stream` -- also inside a stream capture.  Layers of
+ * different lanes overlap on the GPU, which hides the start-up and reduction latency of small layers; every
+ * layer's result is bit for bit that of gaconv_schedule_run_layer.  lanes in 1..8; with lanes > 1 the
+ * descriptors must carry distinct workspaces (GACONV_ERR_BAD_DESC otherwise).  x, dy, dw, descs: host arrays
+ * of num_layers device pointers / descriptor pointers.  Calls on one device share the lanes: enqueueing from
+ * several host threads is serialised. */
+gaconv_status_t gaconv_schedule_run_step(const gaconv_schedule_t *sched, int64_t step, int32_t num_layers,
+                                         const void *const *x, const void *const *dy, float *const *dw,
+                                         const gaconv_conv_desc_t *const *descs, int32_t lanes, void *stream);
 void gaconv_schedule_destroy(gaconv_schedule_t *sched);
 
 #ifdef __cplusplus

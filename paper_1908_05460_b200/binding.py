@@ -32,7 +32,7 @@ SCHED_EVERY_4TH_LAYER, SCHED_ALT_LAYER_ALT_BATCH, SCHED_ALL_LAYERS_EVERY_4TH_BAT
 EXPORTS = [
     "gaconv_status_string", "gaconv_launch_count", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
     "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_poll_async_status",
-    "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_destroy",
+    "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_run_step", "gaconv_schedule_destroy",
     "gaconv_dw_exact_static", "gaconv_static_scratch_bytes", "gaconv_poll_async_status_static", "gaconv_approx_select_topk",
 ]
 
@@ -85,6 +85,8 @@ def load():
     lib.gaconv_schedule_method.argtypes = [vp, i32, ctypes.c_int64]
     lib.gaconv_schedule_method.restype = i32
     lib.gaconv_schedule_run_layer.argtypes = [vp, i32, ctypes.c_int64, vp, vp, vp, dp, vp]
+    lib.gaconv_schedule_run_step.argtypes = [vp, ctypes.c_int64, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                             ctypes.POINTER(dp), i32, vp]
     lib.gaconv_schedule_destroy.argtypes = [vp]
     lib.gaconv_schedule_destroy.restype = None
     _lib = lib
@@ -216,6 +218,18 @@ class Schedule:
     def run_layer(self, layer: int, step: int, x, dy, dw, desc: ConvDesc, stream=None):
         _check(load().gaconv_schedule_run_layer(self._h, layer, step, _ptr(x), _ptr(dy), _ptr(dw), ctypes.byref(desc),
                                                 _stream(stream)), "gaconv_schedule_run_layer")
+
+    def pack_step(self, xs, dys, dws, descs):
+        """Marshal the per-layer arrays of run_step once (the tensors and descriptors must stay alive)."""
+        n = len(descs)
+        VP, DP = ctypes.c_void_p * n, ctypes.POINTER(ConvDesc) * n
+        return (n, VP(*[_ptr(t) for t in xs]), VP(*[_ptr(t) for t in dys]), VP(*[_ptr(t) for t in dws]),
+                DP(*[ctypes.pointer(d) for d in descs]))
+
+    def run_step(self, step: int, packed, lanes: int = 4, stream=None):
+        n, xs, dys, dws, ds = packed
+        _check(load().gaconv_schedule_run_step(self._h, step, n, xs, dys, dws, ds, lanes, _stream(stream)),
+               "gaconv_schedule_run_step")
 
     def close(self):
         if self._h:

@@ -2,6 +2,7 @@
 // approximation-schedule driver (paper Section 2.5).  Every step of the path runs in this library's
 // kernels; there is no CPU or library fallback.
 #include <atomic>
+#include <mutex>
 #include <new>
 
 #include "gaconv_internal.h"
@@ -419,6 +420,77 @@ gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t* s, int32_t la
     if (m == GACONV_METHOD_EXACT) return gaconv_dw_exact(x, dy, dw, desc, stream);
     const uint64_t seed = splitmix64(s->seed ^ splitmix64((uint64_t)step * 0x100000001B3ull + (uint64_t)layer));
     return gaconv_dw_approx(m, x, dy, dw, desc, seed, stream);
+}
+
+// ---- lanes: side streams on which the layers of a step run next to one another ----------------------
+namespace {
+
+constexpr int kMaxLanes = 8, kMaxLaneDevices = 64;
+struct LanePool {
+    bool ready = false;
+    cudaStream_t side[kMaxLanes - 1] = {};
+    cudaEvent_t fork = nullptr, join[kMaxLanes - 1] = {};
+};
+std::mutex g_lane_mutex;
+LanePool g_lanes[kMaxLaneDevices];
+
+// streams and events of the current device, created on first use (host objects; no device memory)
+LanePool* lane_pool()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxLaneDevices) return nullptr;
+    LanePool& p = g_lanes[dev];
+    if (!p.ready) {
+        if (cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int i = 0; i < kMaxLanes - 1; ++i)
+            if (cudaStreamCreateWithFlags(&p.side[i], cudaStreamNonBlocking) != cudaSuccess ||
+                cudaEventCreateWithFlags(&p.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        p.ready = true;
+    }
+    return &p;
+}
+
+}  // namespace
+
+gaconv_status_t gaconv_schedule_run_step(const gaconv_schedule_t* s, int64_t step, int32_t num_layers, const void* const* x,
+                                         const void* const* dy, float* const* dw, const gaconv_conv_desc_t* const* descs,
+                                         int32_t lanes, void* stream)
+{
+    if (s == nullptr || x == nullptr || dy == nullptr || dw == nullptr || descs == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (num_layers < 1 || num_layers > s->num_layers || step < 0 || lanes < 1 || lanes > kMaxLanes) return GACONV_ERR_BAD_DESC;
+    for (int l = 0; l < num_layers; ++l) {
+        if (descs[l] == nullptr) return GACONV_ERR_NULL_POINTER;
+        // layers that run next to one another must not share scratch
+        if (lanes > 1 && descs[l]->workspace != nullptr)
+            for (int o = 0; o < l; ++o)
+                if (descs[o]->workspace == descs[l]->workspace) return GACONV_ERR_BAD_DESC;
+    }
+    cudaStream_t main_stream = static_cast<cudaStream_t>(stream);
+    if (lanes == 1 || num_layers == 1) {
+        for (int l = 0; l < num_layers; ++l) {
+            const gaconv_status_t st = gaconv_schedule_run_layer(s, l, step, x[l], dy[l], dw[l], descs[l], stream);
+            if (st != GACONV_OK) return st;
+        }
+        return GACONV_OK;
+    }
+    std::lock_guard<std::mutex> lock(g_lane_mutex);          // one set of lanes per device: enqueueing is serialised
+    LanePool* pool = lane_pool();
+    if (pool == nullptr) return GACONV_ERR_CUDA;
+    const int used = lanes < num_layers ? lanes : num_layers;
+    // fork: the side streams start after everything already enqueued on the caller's stream
+    if (cudaEventRecord(pool->fork, main_stream) != cudaSuccess) return GACONV_ERR_CUDA;
+    for (int i = 0; i < used - 1; ++i)
+        if (cudaStreamWaitEvent(pool->side[i], pool->fork, 0) != cudaSuccess) return GACONV_ERR_CUDA;
+    gaconv_status_t result = GACONV_OK;
+    for (int l = 0; l < num_layers && result == GACONV_OK; ++l) {
+        const int lane = l % used;
+        result = gaconv_schedule_run_layer(s, l, step, x[l], dy[l], dw[l], descs[l], lane == 0 ? stream : static_cast<void*>(pool->side[lane - 1]));
+    }
+    // join (also after an error, so that the side streams never stay forked from a capturing stream)
+    for (int i = 0; i < used - 1; ++i)
+        if (cudaEventRecord(pool->join[i], pool->side[i]) != cudaSuccess || cudaStreamWaitEvent(main_stream, pool->join[i], 0) != cudaSuccess)
+            return GACONV_ERR_CUDA;
+    return result;
 }
 
 void gaconv_schedule_destroy(gaconv_schedule_t* s)

@@ -506,3 +506,44 @@ def test_rsck_output_layout(li):
         z = oracle.dw_random(ref.size, 3, 1.0 / 128).reshape(ref.shape)
         assert np.max(np.abs(g.approx(B.METHOD_RANDOM, seed=3) - z)) <= 1e-5 * 6 / 128
         assert np.all(g.approx(B.METHOD_ZERO) == 0)
+
+
+# ---- a whole step on several lanes: every layer's dW is bit for bit the per-layer call's ----
+def test_run_step_on_lanes_equals_per_layer_calls():
+    layers = [SMALL[0], SMALL[2], SMALL[8], SMALL[9], TC_SHAPES[4], SMALL[5], TC_SHAPES[14], SMALL[12]]
+    gs = []
+    for li, layer in enumerate(layers):
+        x, dy = _inputs(layer, torch.bfloat16, 800 + li)
+        gs.append(GpuLayer(layer, torch.bfloat16, x, dy, alpha=0.5))
+    sched = B.Schedule(len(gs), B.SCHED_EVERY_4TH_LAYER, B.METHOD_TOP1)           # layers 2 and 6 (1-based) approximated
+    want = []
+    for li, g in enumerate(gs):
+        g.dw.fill_(float("nan"))
+        sched.run_layer(li, 5, g.x, g.dy, g.dw, g.desc)
+        want.append(g.logical_dw())
+    assert [sched.method(l, 5) for l in range(len(gs))].count(B.METHOD_TOP1) == 2
+    packed = sched.pack_step([g.x for g in gs], [g.dy for g in gs], [g.dw for g in gs], [g.desc for g in gs])
+    for lanes in (1, 3, 8):
+        for g in gs:
+            g.dw.fill_(float("nan"))
+        sched.run_step(5, packed, lanes=lanes)
+        for li, g in enumerate(gs):
+            np.testing.assert_array_equal(g.logical_dw(), want[li])
+    # inside a stream capture the fork and join of the lanes are part of the graph
+    for g in gs:
+        g.dw.fill_(float("nan"))
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr):
+        sched.run_step(5, packed, lanes=4)
+    for g in gs:
+        g.dw.fill_(float("nan"))
+    gr.replay()
+    for li, g in enumerate(gs):
+        np.testing.assert_array_equal(g.logical_dw(), want[li])
+        assert B.gaconv_poll_async_status(g.desc) == B.OK
+    # layers that run next to one another may not share a workspace
+    shared = sched.pack_step([gs[0].x, gs[0].x], [gs[0].dy, gs[0].dy], [gs[0].dw, gs[1].dw], [gs[0].desc, gs[0].desc])
+    with pytest.raises(B.GaconvError) as e:
+        sched.run_step(5, shared, lanes=2)
+    assert e.value.status == B.ERR_BAD_DESC
