@@ -299,7 +299,13 @@ def main():
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
     ap.add_argument("--layer-iters", type=int, default=5, help="per-layer timing repetitions (median)")
-    ap.add_argument("--lanes", type=int, default=4, help="streams on which the layers of a step run next to one another (1..8)")
+    ap.add_argument("--lanes", type=int, default=8, help="streams on which the layers of a step run next to one another (1..8)")
+    ap.add_argument("--budget-div", type=float, default=12.0, help="SM share of a layer in the step: 148 * roofline us / this")
+    ap.add_argument("--budget-min", type=int, default=18)
+    ap.add_argument("--budget-max", type=int, default=74)
+    ap.add_argument("--allreduce", action="store_true",
+                    help="N > 1: treat the ranks' batches as shards of one batch and sum the exact / top-1 filter gradients of the "
+                         "layer set over the ranks in one bucketed all-reduce per step (inside the timed region)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -358,9 +364,16 @@ def main():
                 s.x = s.x_host.cuda(); s.dy = s.dy_host.cuda()
                 s.dw = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32, device="cuda")
                 s.dw_host = torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32).pin_memory()
-                s.desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n)
-                s.ws = B.attach_workspace(s.desc)
                 s.eb = 2 if s.dtype == torch.bfloat16 else 4
+                s.desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n)            # per-layer timings: the whole GPU for one layer
+                s.ws = B.attach_workspace(s.desc)
+                # the step runs layers next to one another on several lanes: each layer is sized for a share of the SMs
+                # that grows with its roofline time (18 SMs for the latency-bound layers, up to half the GPU)
+                t_roof = max(l.flops_exact() / (peaks["bf16_tflops"] * 1e12 * (1.0 if s.eb == 2 else 0.5)),
+                             l.bytes_exact(s.eb) / (peaks["hbm_gbs"] * 1e9)) * 1e6
+                s.budget = 0 if args.lanes == 1 else max(args.budget_min, min(args.budget_max, int(148 * t_roof / args.budget_div)))
+                s.step_desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n, sm_budget=s.budget)
+                s.step_ws = B.attach_workspace(s.step_desc)
                 h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs
                 d2h += 4 * s.dw.numel() * 4
                 slots.append(s)
@@ -377,7 +390,7 @@ def main():
     def run_one(s, m, t):
         scheds[m].run_layer(s.sid, 4 * t + (3 if m >= 0 else 0), s.x, s.dy, s.dw, s.desc)
 
-    packed = {m: scheds[m].pack_step([s.x for s in slots], [s.dy for s in slots], [s.dw for s in slots], [s.desc for s in slots])
+    packed = {m: scheds[m].pack_step([s.x for s in slots], [s.dy for s in slots], [s.dw for s in slots], [s.step_desc for s in slots])
               for _, m in methods}
 
     def step(t):
@@ -399,7 +412,14 @@ def main():
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             step(1)
-    run_step = (lambda t: graph.replay()) if graph is not None else step
+    base_step = (lambda t: graph.replay()) if graph is not None else step
+    if args.allreduce and world > 1:
+        # data-parallel filter gradient: after the step every rank holds the gradient of its shard; one bucket, one sum
+        def run_step(t):
+            base_step(t)
+            dist_util.allreduce_dw_bucket([s.dw for s in slots], [B.METHOD_EXACT] * len(slots))
+    else:
+        run_step = base_step
     for t in range(args.warmup):
         run_step(t)
     barrier()
@@ -423,6 +443,26 @@ def main():
     ms_step = dist_util.max_over_ranks(ms_total, "cuda") / args.steps      # slowest rank decides
     passes = len(slots)
     value = dist_util.us_per_layer(ms_step, passes, world)
+
+    # ---- the step, method by method: one graph per method, replayed over cold inputs (another method's pass in between) ----
+    es0, ee0 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_by_method = {}
+    if not args.no_graph and args.layer_iters > 0:
+        gm = {}
+        for name, m in methods:
+            gm[name] = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gm[name]):
+                scheds[m].run_step(4 * 1 + (3 if m >= 0 else 0), packed[m], lanes=args.lanes)
+        order = [n for n, _ in methods]
+        ts = {n: [] for n in order}
+        for rep in range(4):
+            for i, name in enumerate(order):
+                gm[order[(i + 1) % 2]].replay()            # stream the other input-reading method's data through L2 first
+                es0.record(); gm[name].replay(); ee0.record(); ee0.synchronize()
+                if rep > 0:
+                    ts[name].append(es0.elapsed_time(ee0) * 1e3)
+        step_by_method = {n: statistics.median(v) for n, v in ts.items()}
+        del gm
 
     # ---- per-layer timing on the launching stream ----
     # streamed: a CUDA graph of back-to-back launches of one layer, each on its own copy of the inputs,
@@ -564,11 +604,14 @@ def main():
                                % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), passes,
                                   ", ".join("%s %s" % ({2: "resnet20", 3: "cnn2", 4: "vgg19"}[c], "/".join(dn)) for c, _, dn in sets)),
                    "layer_passes_per_step": passes, "cuda_graph": graph is not None, "lanes": args.lanes,
+                   "parallelism": ("dp%d, one dW all-reduce per step" % world) if (args.allreduce and world > 1) else ("%d independent replicas" % world if world > 1 else "1 GPU"),
+                   "sm_budget": "per layer min(%d, max(%d, 148 * roofline us / %g)) SMs in the step; whole GPU in the per-layer timings"
+                                % (args.budget_max, args.budget_min, args.budget_div),
                    "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
                          "order); per-layer timings stream over rotating input copies > 2.5x L2" % (input_bytes / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
-        "breakdown_us": {"streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
+        "breakdown_us": {"step_by_method": step_by_method, "streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
                          "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
                          "top1_speedup_over_exact": (sum_us["exact"] / sum_us["top1"]) if table else None,
                          "per_set": nets},

@@ -70,6 +70,11 @@ typedef struct gaconv_conv_desc {
     int32_t  math;                     /* gaconv_math_t                                                   */
     int32_t  algo;                     /* gaconv_algo_t                                                   */
     int32_t  topk;                     /* GACONV_METHOD_TOPK: entries retained per map, 1..GACONV_MAX_TOPK (else ignored) */
+    int32_t  sm_budget;                /* 0: size every launch for the whole GPU (lowest latency of a single layer);
+                                          n > 0: size it for about n SMs, so that layers running next to one another
+                                          (gaconv_schedule_run_step with several lanes) share the GPU instead of
+                                          queueing for it.  Part of the problem statement: it changes how the
+                                          reduction is split, hence the rounding, never the exact value             */
     float    alpha;                    /* dw = alpha * (...); 1 for parity, 1/128 in the paper's runs (Section 2.3) */
     float    rand_std;                 /* METHOD_RANDOM: standard deviation; the paper uses 1/128 (Section 2.2)     */
     void    *workspace;                /* device scratch prepared by gaconv_workspace_init                */

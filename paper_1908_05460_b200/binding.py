@@ -40,7 +40,7 @@ EXPORTS = [
 class ConvDesc(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32)] + \
         [(f, ctypes.c_int32) for f in ("n", "c", "h", "w", "k", "r", "s", "stride_h", "stride_w", "pad_h", "pad_w",
-                                       "in_dtype", "x_layout", "dy_layout", "dw_layout", "math", "algo", "topk")] + \
+                                       "in_dtype", "x_layout", "dy_layout", "dw_layout", "math", "algo", "topk", "sm_budget")] + \
         [("alpha", ctypes.c_float), ("rand_std", ctypes.c_float),
          ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
@@ -123,7 +123,7 @@ def _stream(stream):
 
 
 def make_desc(layer: ConvLayer, dtype: torch.dtype, *, x_layout=X_NHWC, dw_layout=DW_KRSC, alpha=1.0,
-              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO, topk=1) -> ConvDesc:
+              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO, topk=1, sm_budget=0) -> ConvDesc:
     d = ConvDesc()
     d.struct_size = ctypes.sizeof(ConvDesc)
     d.n, d.c, d.h, d.w, d.k, d.r, d.s = layer.n, layer.c, layer.h, layer.w, layer.k, layer.r, layer.s
@@ -131,7 +131,7 @@ def make_desc(layer: ConvLayer, dtype: torch.dtype, *, x_layout=X_NHWC, dw_layou
     d.pad_h = d.pad_w = layer.pad
     d.in_dtype = BF16 if dtype == torch.bfloat16 else F32
     d.x_layout, d.dy_layout, d.dw_layout = x_layout, DY_NKPQ, dw_layout
-    d.math, d.algo, d.topk = math, algo, topk
+    d.math, d.algo, d.topk, d.sm_budget = math, algo, topk, sm_budget
     d.alpha, d.rand_std = alpha, rand_std
     d.workspace, d.workspace_bytes = None, 0
     return d

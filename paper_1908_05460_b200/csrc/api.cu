@@ -50,6 +50,8 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     }
     g->bf16 = d->in_dtype == GACONV_BF16;
     g->alpha = d->alpha;
+    if (d->sm_budget < 0) return GACONV_ERR_BAD_DESC;
+    g->sm_budget = d->sm_budget;
     return GACONV_OK;
 }
 

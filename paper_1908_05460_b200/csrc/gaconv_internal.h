@@ -62,6 +62,7 @@ struct Geom {
     long long ws_k, ws_c, ws_r, ws_s;   // element strides of dW
     bool bf16;
     float alpha;
+    int sm_budget;                      // 0: plan for the whole GPU; n > 0: for about n SMs
 };
 
 // ---- fixed-order sum of split partials: dw = alpha * sum_sp partial[sp][0..count) ----

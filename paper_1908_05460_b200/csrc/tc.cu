@@ -754,9 +754,11 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // second kernel adds them up.  Larger clusters mean less workspace traffic, but fewer resident CTAs (clusters
     // are placed GPC by GPC: 148 CTAs fit as pairs, 135 as triples, 132 as quadruples).
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
+    // SMs this launch may count on: all of them, or the caller's budget (layers sharing the GPU on several lanes)
+    const int sms = g.sm_budget > 0 ? std::min(g.sm_budget, sm_count()) : sm_count();
     int max_splits = env_int("GACONV_TC_SPLITS", 0);
     if (max_splits <= 0) {
-        max_splits = sm_count() / tiles;
+        max_splits = sms / tiles;
         if (max_splits < 1) max_splits = 1;
     }
     if (max_splits > P.chunks) max_splits = P.chunks;
@@ -767,7 +769,8 @@ bool plan_tc(const Geom& g, TcPlan* out)
     int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0}, most = 0;
     for (int c = 1; c <= 4; ++c) {
         if (c > cl_cap || c > max_splits || (cl_force && c != cl_force)) continue;
-        per_of[c] = std::min(max_splits / c, resident_clusters(c) / tiles);               // clusters per tile
+        // clusters per tile: within the split budget and, where the tiles allow it, within one resident wave
+        per_of[c] = std::min(max_splits / c, std::max(1, std::min(resident_clusters(c), std::max(1, sms / c)) / tiles));
         sp_of[c] = per_of[c] * c;
         most = std::max(most, sp_of[c]);
     }

@@ -547,3 +547,39 @@ def test_run_step_on_lanes_equals_per_layer_calls():
     with pytest.raises(B.GaconvError) as e:
         sched.run_step(5, shared, lanes=2)
     assert e.value.status == B.ERR_BAD_DESC
+
+
+# ---- training-step integration: forward and input gradient from the framework, filter gradient from the library ----
+def test_autograd_module_matches_the_frameworks_filter_gradient_and_follows_the_schedule():
+    from paper_1908_05460_b200.autograd import GAConv2d
+    torch.manual_seed(3)
+    torch.backends.cudnn.allow_tf32 = False          # the framework's convolutions in true fp32, so that they can serve as a reference
+    sched = B.Schedule(2, B.SCHED_LAYER2_ALT_BATCH, B.METHOD_TOP1)                # layer 2 approximated on odd steps
+    conv1 = GAConv2d(3, 16, 3, padding=1, schedule=sched, layer_index=0)
+    conv2 = GAConv2d(16, 16, 3, stride=2, padding=1, schedule=sched, layer_index=1)
+    x = torch.randn(8, 3, 32, 32, device="cuda")
+    for step in (0, 1):
+        conv1.step = conv2.step = step
+        for m in (conv1, conv2):
+            m.weight.grad = None
+        xin = x.clone().requires_grad_(True)
+        h = torch.relu(conv1(xin))
+        y = conv2(h)
+        g = torch.randn_like(y)
+        y.backward(g)
+        # the framework's own gradients of the same graph
+        w1 = conv1.weight.detach().clone().requires_grad_(True); w2 = conv2.weight.detach().clone().requires_grad_(True)
+        xr = x.clone().requires_grad_(True)
+        hr = torch.relu(torch.nn.functional.conv2d(xr, w1, None, 1, 1))
+        yr = torch.nn.functional.conv2d(hr, w2, None, 2, 1)
+        yr.backward(g)
+        assert torch.allclose(xin.grad, xr.grad, rtol=1e-3, atol=1e-4)             # input gradients: framework both times
+        assert torch.allclose(conv1.weight.grad, w1.grad, rtol=1e-3, atol=1e-3)    # layer 1 is always exact
+        if step == 0:
+            assert torch.allclose(conv2.weight.grad, w2.grad, rtol=1e-3, atol=1e-3)
+        else:                                                                      # odd step: Algorithm 1 on layer 2
+            layer = ConvLayer("l2", 8, 16, 32, 32, 16, 3, 3, 2, 1)
+            ref, dn = oracle.dw_top1(to_f64(hr.detach().cpu()), to_f64(g.cpu()), oshape(layer))
+            got = conv2.weight.grad.double().cpu().numpy()
+            assert norm_err(got, ref, dn) <= 1e-4        # torch's forward runs in TF32/fp32: the activations differ in the last bits
+            assert not torch.allclose(conv2.weight.grad, w2.grad, rtol=1e-2, atol=1e-3)
