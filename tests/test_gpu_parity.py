@@ -45,6 +45,7 @@ SMALL = [
     ConvLayer("4x4", 8, 48, 4, 4, 80, 3, 3, 1, 1),
     ConvLayer("8x8", 8, 64, 8, 8, 64, 3, 3, 1, 1),
     ConvLayer("8x8 c128 (top-1 via sparse dY + dense kernel)", 6, 128, 8, 8, 96, 3, 3, 1, 1),
+    ConvLayer("8x8 c256 k40 n19 (top-1 via sparse dY + dense kernel, ragged)", 19, 256, 8, 8, 40, 3, 3, 1, 1),
     ConvLayer("4x4 c256", 5, 256, 4, 4, 64, 3, 3, 1, 1),
     ConvLayer("1x1", 4, 20, 9, 9, 12, 1, 1, 1, 0, dy_std=1.0),
     ConvLayer("7x7 filter", 2, 5, 12, 12, 6, 7, 7, 1, 3, dy_std=1.0),
