@@ -132,6 +132,8 @@ struct TcPlan {
     alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
 };
 bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel
+// fp32 inputs on the same kernel with TF32 MMAs: passes = 3 (split operands, fp32 accuracy) or 1 (plain TF32)
+bool plan_tc_f32(const Geom& g, int passes, TcPlan* plan);
 // dy == nullptr: the scratch already holds the transposed operand (plan.reads_transposed_dy only)
 cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* counters,
                       uint32_t* status,

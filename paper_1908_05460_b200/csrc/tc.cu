@@ -71,6 +71,15 @@ __device__ __forceinline__ float4 ld_dsmem_f4(uint32_t local_addr, uint32_t rank
     asm("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote));
     return v;
 }
+// fp32 operands read as TF32 (the tensor core takes the upper 19 bits of each word)
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -107,6 +116,13 @@ struct TcParams {
                         //    rows), as the wide tile does for maps of 64 pixels and more
     int b_lbo;          // B descriptor: bytes between the column-shift atoms of an MMA
     int b_sub_bytes;    // B descriptor advance from one A box (or image row) to the next
+    int f32;            // 1: fp32 inputs on kind::tf32 MMAs (32-pixel A boxes, 32-channel B tiles, k-steps of 8 pixels).
+                        //    passes == 3: the operands come as two planes each, big = the TF32 part of x and small = x - big,
+                        //    and every k-step issues big*big + big*small + small*big into the same accumulator (fp32 accuracy);
+                        //    passes == 1: the tensors themselves, cut to TF32 by the tensor core
+    int passes;
+    int kpx;            // pixels per k-step: 16 (bf16) or 8 (tf32)
+    int a_plane_bytes, b_plane_bytes;   // distance from the big to the small plane inside a stage
     int by_image;       // 1: a chunk is ci whole images (maps under 64 pixels)
     int a_k4_step;      // descriptor advance (16-byte units) from one k-step to the next inside an A box
     int a_lbo;          // leading byte offset of the A descriptor
@@ -205,8 +221,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const int cpi = whole_maps ? 1 : g.p / P.bp;
         if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
-        const uint32_t tx_bytes = (P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes;
-        const int n_a = P.tiny ? P.m / 64 : P.by_image ? 1 : P.a_subs, n_all = n_a + P.b_tiles;
+        const int planes = P.f32 && P.passes == 3 ? 2 : 1;
+        const uint32_t tx_bytes = planes * ((P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes);
+        const int n_a = P.f32 ? planes * P.a_subs : P.tiny ? P.m / 64 : P.by_image ? 1 : P.a_subs, n_all = n_a + planes * P.b_tiles;
         // what copy `lane` is: image and box of an A copy, or filter row and column shift of a B copy
         const int a_img = (P.tiny || P.by_image) ? 0 : lane / P.a_subs_img, a_sub = (P.tiny || P.by_image) ? 0 : lane - a_img * P.a_subs_img;
         const int b_idx = lane - n_a, b_rr = b_idx > 0 ? b_idx / g.s : 0, b_ss = b_idx > 0 ? b_idx - b_rr * g.s : 0;
@@ -224,7 +241,15 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             const uint32_t sa = smem_base + st * P.stage_bytes;
             const uint32_t sb = sa + P.a_region_bytes;
             for (int b = lane; b < n_all; b += 32) {
-                if (b < n_a) {
+                if (P.f32) {                                                     // fp32: boxes of 32 pixels, one set per plane
+                    if (b < n_a) {
+                        const int pl = b / P.a_subs, sub = b - pl * P.a_subs, i = sub / P.a_subs_img, sb_ = sub - i * P.a_subs_img;
+                        tma_load_4d(sa + pl * P.a_plane_bytes + sub * P.a_sub_bytes, &map_dy, full, p0 * g.q + P.a_sub_px * sb_, k0, n0 + i, pl);
+                    } else {
+                        const int pl = b - n_a;
+                        tma_load_5d(sb + pl * P.b_plane_bytes, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0, pl);
+                    }
+                } else if (b < n_a) {
                     if (P.tiny2) {                                               // one box per 64-channel atom, [pixel][image][k]
                         tma_load_3d(sa + b * P.a_lbo, &map_dy, full, k0 + 64 * b, n0, 0);
                     } else if (P.tiny) {                                         // one box per 64-channel atom, [image][pixel][k]
@@ -261,14 +286,16 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const int issuer = warp - 1;
         // ------------------------------------------------------------------ MMA issuer
         // descriptors are assembled from a constant high word and a low word that only advances
-        const uint32_t a_row_bytes = P.tiny ? 128u : P.a_sub_px * 2, b_row_bytes = P.ct * 2;
+        const uint32_t eb = P.f32 ? 4u : 2u;
+        const uint32_t a_row_bytes = P.tiny ? 128u : P.a_sub_px * eb, b_row_bytes = P.ct * eb;
         const uint32_t a_hi = ((8 * a_row_bytes) >> 4) | (1u << 14) | ((uint32_t)P.a_swz << 29);
         const uint32_t wt = g.q + g.s - 1;                       // pixels per tile row in wide mode
         // stride between the two 8-pixel halves of a k-step: contiguous, except in wide mode when a k-step spans two rows
-        const uint32_t b_sbo = (P.wide && g.q == 8) ? wt * b_row_bytes : 8 * b_row_bytes;
+        // (fp32: an MN-major tf32 operand uses the 128-byte swizzle on 32-byte units, whose K groups are 4 pixels)
+        const uint32_t b_sbo = P.f32 ? 4 * b_row_bytes : (P.wide && g.q == 8) ? wt * b_row_bytes : 8 * b_row_bytes;
         const uint32_t b_hi = (b_sbo >> 4) | (1u << 14) | ((uint32_t)P.b_swz << 29);
         const uint32_t a_lo_c = (((uint32_t)P.a_lbo >> 4) & 0x3fffu) << 16, b_lo_c = (((uint32_t)P.b_lbo >> 4) & 0x3fffu) << 16;
-        const int ks_per_sub = P.a_sub_px / 16;
+        const int ks_per_sub = P.a_sub_px / P.kpx;
         const uint32_t a_k4 = (uint32_t)P.a_k4_step;
         const uint32_t a_sub_step = (uint32_t)P.a_sub_bytes >> 4;
         const uint32_t b_r_step = (P.wide ? wt * b_row_bytes : P.halo ? (uint32_t)g.q * b_row_bytes : (uint32_t)g.s * P.b_tile_stride) >> 4;
@@ -276,7 +303,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         uint32_t b_k_off[4];
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4)
-            b_k_off[k4] = (P.wide ? (((16u * k4) / g.q) * wt + (16u * k4) % g.q) * b_row_bytes : 16u * k4 * b_row_bytes) >> 4;
+            b_k_off[k4] = (P.wide ? ((((uint32_t)P.kpx * k4) / g.q) * wt + ((uint32_t)P.kpx * k4) % g.q) * b_row_bytes : (uint32_t)P.kpx * k4 * b_row_bytes) >> 4;
         const uint32_t b_sub_step = (uint32_t)P.b_sub_bytes >> 4;
         const int R = R_T ? R_T : P.rc;
         const int KS = KS_T ? KS_T : ks_per_sub;
@@ -294,6 +321,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         const uint64_t a_hi64 = (uint64_t)a_hi << 32, b_hi64 = (uint64_t)b_hi << 32;
         const uint32_t idesc = P.idesc;
         const int mine = P.dual ? issuer : 0, it_step_mask = P.dual ? 1 : 0;
+        const uint32_t a_small = (uint32_t)P.a_plane_bytes >> 4, b_small = (uint32_t)P.b_plane_bytes >> 4;      // fp32, three passes
         int st = 0, ph = 0;
         bool fresh = true;            // the next k-step starts the accumulation (overwrites TMEM)
         for (int it = 0; it < nchunks; ++it) {
@@ -305,6 +333,23 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                 // 14-bit start-address fields: in a cluster launch shared addresses carry the CTA rank in high bits
                 uint32_t a_lo = a_lo_c | ((sa >> 4) & 0x3fffu);
                 uint32_t b_lo = b_lo_c | (((sa + P.a_region_bytes) >> 4) & 0x3fffu);
+                if (P.f32) {
+                    // fp32 inputs: one accumulator per issuer (dual), k-steps of eight pixels; with split operands
+                    // big*big, then the two cross terms, every k-step
+                    for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step, b_lo += b_sub_step) {
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            if (k4 >= KS) break;
+                            const uint64_t ad = a_hi64 | (a_lo + a_k4 * k4), bd = b_hi64 | (b_lo + b_k_off[k4]);
+                            umma_tf32(d_row[0], ad, bd, idesc, fresh ? 0u : 1u);
+                            fresh = false;
+                            if (P.passes == 3) {
+                                umma_tf32(d_row[0], ad, bd + b_small, idesc, 1u);
+                                umma_tf32(d_row[0], ad + a_small, bd, idesc, 1u);
+                            }
+                        }
+                    }
+                } else
                 for (int sub = 0; sub < P.a_subs; ++sub, a_lo += a_sub_step) {
                     if (fresh) {      // first k-step of this accumulator: accumulate flag off
 #pragma unroll
@@ -574,6 +619,26 @@ reduce_slots_kernel(const float4* __restrict__ partial, float* __restrict__ dw, 
     }
 }
 
+// fp32 operand -> two planes: big = x with the 13 low mantissa bits cleared (exactly a TF32 number) and
+// small = x - big (exact in fp32; at most 13 significant bits, of which the tensor core keeps 11).  Then
+// a*b = big_a*big_b + big_a*small_b + small_a*big_b up to ~2^-21 |a*b|.
+__global__ void __launch_bounds__(256)
+split_tf32_kernel(const float4* __restrict__ src, float4* __restrict__ big, float4* __restrict__ small, size_t nvec)
+{
+    pdl_release_next_grid();
+    pdl_wait_prior_grid();
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        const float4 v = __ldg(src + i);
+        float4 b, sm;
+        b.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); sm.x = v.x - b.x;
+        b.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); sm.y = v.y - b.y;
+        b.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); sm.z = v.z - b.z;
+        b.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); sm.w = v.w - b.w;
+        big[i] = b; small[i] = sm;
+    }
+}
+
 // ---------------------------------------------------------------- host side
 CUtensorMapSwizzle swizzle_for(int bytes) {
     return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
@@ -625,6 +690,47 @@ int resident_clusters(int cl)
     return cached[dev][cl];
 }
 
+// Splits of the reduction and cluster size for `tiles` output tiles (fills P.cl, P.splits, P.chunk_base, P.chunk_rem).
+bool choose_splits(TcParams& P, const Geom& g, int tiles)
+{
+    // Splits of the reduction: one wave of CTAs, one per SM.  Consecutive splits form a thread-block cluster of up
+    // to 4 that reduces through distributed shared memory; the clusters of a tile meet in the workspace, where the
+    // second kernel adds them up.  Larger clusters mean less workspace traffic, but fewer resident CTAs (clusters
+    // are placed GPC by GPC: 148 CTAs fit as pairs, 135 as triples, 132 as quadruples).
+    // SMs this launch may count on: all of them, or the caller's budget (layers sharing the GPU on several lanes)
+    const int sms = g.sm_budget > 0 ? std::min(g.sm_budget, sm_count()) : sm_count();
+    int max_splits = env_int("GACONV_TC_SPLITS", 0);
+    if (max_splits <= 0) {
+        max_splits = sms / tiles;
+        if (max_splits < 1) max_splits = 1;
+    }
+    if (max_splits > P.chunks) max_splits = P.chunks;
+    const int cl_cap = env_int("GACONV_TC_CLUSTER", 4);
+    // Measured on the layer shapes of the three networks: a cluster whose splits cover the whole tile (no workspace,
+    // no second kernel) wins even at two thirds of the CTAs; otherwise the largest cluster that keeps 85% of them.
+    const int cl_force = env_int("GACONV_TC_FORCE_CL", 0);
+    int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0}, most = 0;
+    for (int c = 1; c <= 4; ++c) {
+        if (c > cl_cap || c > max_splits || (cl_force && c != cl_force)) continue;
+        // clusters per tile: within the split budget and, where the tiles allow it, within one resident wave
+        per_of[c] = std::min(max_splits / c, std::max(1, std::min(resident_clusters(c), std::max(1, sms / c)) / tiles));
+        sp_of[c] = per_of[c] * c;
+        most = std::max(most, sp_of[c]);
+    }
+    int cl = 0, splits = 0;
+    for (int c = 4; c >= 1 && cl == 0; --c)
+        if (per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
+    for (int c = 4; c >= 1 && cl == 0; --c)
+        if (sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
+    if (cl == 0) return false;
+    P.cl = cl;
+    P.splits = splits;
+    P.reduce_parts = std::max(1, 2 * sm_count() / tiles);
+    P.chunk_base = P.chunks / splits;
+    P.chunk_rem = P.chunks - P.chunk_base * splits;
+    return true;
+}
+
 }  // namespace
 
 bool plan_tc(const Geom& g, TcPlan* out)
@@ -662,6 +768,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.dual = (P.rc == 1 && env_int("GACONV_TC_DUAL", 1)) ? 1 : 0;
     P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     P.tiny = tiny ? 1 : 0;
+    P.kpx = 16; P.passes = 1;
     P.by_image = small_map ? 1 : 0;
     // channels per tile: one swizzle span wide (16, 32 or 64 channels), limited by MMA N <= 256 and TMEM columns
     int ct = g.c >= 64 ? 64 : g.c >= 32 ? 32 : 16;
@@ -749,43 +856,9 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B MN-major, N, M
     P.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((tiny ? 1u : 0u) << 15) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
 
-    // Splits of the reduction: one wave of CTAs, one per SM.  Consecutive splits form a thread-block cluster of up
-    // to 4 that reduces through distributed shared memory; the clusters of a tile meet in the workspace, where the
-    // second kernel adds them up.  Larger clusters mean less workspace traffic, but fewer resident CTAs (clusters
-    // are placed GPC by GPC: 148 CTAs fit as pairs, 135 as triples, 132 as quadruples).
     const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
-    // SMs this launch may count on: all of them, or the caller's budget (layers sharing the GPU on several lanes)
-    const int sms = g.sm_budget > 0 ? std::min(g.sm_budget, sm_count()) : sm_count();
-    int max_splits = env_int("GACONV_TC_SPLITS", 0);
-    if (max_splits <= 0) {
-        max_splits = sms / tiles;
-        if (max_splits < 1) max_splits = 1;
-    }
-    if (max_splits > P.chunks) max_splits = P.chunks;
-    const int cl_cap = env_int("GACONV_TC_CLUSTER", 4);
-    // Measured on the layer shapes of the three networks: a cluster whose splits cover the whole tile (no workspace,
-    // no second kernel) wins even at two thirds of the CTAs; otherwise the largest cluster that keeps 85% of them.
-    const int cl_force = env_int("GACONV_TC_FORCE_CL", 0);
-    int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0}, most = 0;
-    for (int c = 1; c <= 4; ++c) {
-        if (c > cl_cap || c > max_splits || (cl_force && c != cl_force)) continue;
-        // clusters per tile: within the split budget and, where the tiles allow it, within one resident wave
-        per_of[c] = std::min(max_splits / c, std::max(1, std::min(resident_clusters(c), std::max(1, sms / c)) / tiles));
-        sp_of[c] = per_of[c] * c;
-        most = std::max(most, sp_of[c]);
-    }
-    int cl = 0, splits = 0;
-    for (int c = 4; c >= 1 && cl == 0; --c)
-        if (per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
-    for (int c = 4; c >= 1 && cl == 0; --c)
-        if (sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
-    const double best = cl == 0 ? 1e30 : 0.0;
-    if (best == 1e30) return false;
-    P.cl = cl;
-    P.splits = splits;
-    P.reduce_parts = std::max(1, 2 * sm_count() / tiles);
-    P.chunk_base = P.chunks / splits;
-    P.chunk_rem = P.chunks - P.chunk_base * splits;
+    if (!choose_splits(P, g, tiles)) return false;
+    const int splits = P.splits, cl = P.cl;
     // the reduction block must fit the dynamic shared memory (it reuses the operand stages)
     const size_t red_bytes = (size_t)P.m * (P.rc * g.s * ct + 4) * 4;
     if (red_bytes > 212 * 1024) return false;
@@ -806,6 +879,83 @@ bool plan_tc(const Geom& g, TcPlan* out)
     return encode_fn() != nullptr;
 }
 
+// fp32 inputs on the tcgen05 path (kind::tf32): single-row CTAs with the wide X tile, stride 1, rows of 8, 16 or 32
+// output pixels.  passes = 3 (fp32 accuracy through split operands) or 1 (plain TF32).
+bool plan_tc_f32(const Geom& g, int passes, TcPlan* out)
+{
+    if (g.bf16 || g.xs_c != 1 || g.c % 32 != 0) return false;
+    if (g.stride_h != 1 || g.stride_w != 1 || g.r > 7 || g.s > 7 || g.s * 32 > 256) return false;
+    const int pq = g.p * g.q;
+    if (pq % 32 != 0 || g.q % 8 != 0 || 32 % g.q != 0) return false;          // a 32-pixel box is whole rows, a k-step lies in a row
+    if ((size_t)g.n * g.c * g.h * g.w % 4 != 0 || (size_t)g.n * g.k * pq % 4 != 0) return false;
+    TcParams P{};
+    P.g = g;
+    P.f32 = 1; P.passes = passes; P.kpx = 8;
+    P.m = g.k <= 64 ? 64 : 128;
+    P.rsplit = g.r > 1 ? 1 : 0;
+    P.rc = 1; P.dual = 1; P.issuers = 2;
+    P.kb = g.k < P.m ? (g.k + 7) / 8 * 8 : P.m;
+    const int ct = 32;
+    P.ct = ct; P.ct_shift = 5;
+    P.tiles_k = (g.k + P.m - 1) / P.m;
+    P.tiles_c = (g.c + ct - 1) / ct;
+    P.wide = 1; P.b_tiles = 1;
+    P.a_sub_px = 32;
+    P.a_swz = swz_code(128); P.b_swz = 1;               // B: 128-byte swizzle with 32-byte base (MN-major 32-bit elements)
+    const int planes = passes == 3 ? 2 : 1;
+    const int budget = env_int("GACONV_TC_STAGE_KB", 64) * 1024, wt = g.q + g.s - 1;
+    auto stage = [&](int ci, int bp, int* a_bytes, int* tile_bytes) {
+        *a_bytes = (ci * bp * g.q / 32 * P.kb * 128 + 1023) / 1024 * 1024;
+        *tile_bytes = (ci * bp * wt * ct * 4 + 1023) / 1024 * 1024;
+        return planes * (*a_bytes + *tile_bytes);
+    };
+    int ci = 1, bp = 32 / g.q, ab, tb;
+    while (bp * 2 <= g.p && g.p % (bp * 2) == 0 && bp * 2 <= 256 && stage(1, bp * 2, &ab, &tb) <= budget) bp *= 2;
+    if (g.p % bp != 0) return false;
+    if (bp == g.p)
+        while (ci * 2 <= 8 && ci * 2 <= g.n && stage(ci * 2, bp, &ab, &tb) <= budget) ci *= 2;
+    P.ci = ci; P.bp = bp;
+    P.stage_bytes = stage(ci, bp, &ab, &tb);
+    P.a_subs = ci * bp * g.q / 32;
+    P.a_subs_img = P.a_subs / ci;
+    P.a_sub_bytes = P.kb * 128;
+    P.a_k4_step = 2;                                    // eight fp32 pixels = 32 bytes
+    P.a_lbo = 16;
+    P.a_region_bytes = planes * ab;
+    P.a_plane_bytes = ab; P.b_plane_bytes = tb;
+    P.b_tile_bytes = ci * bp * wt * ct * 4; P.b_tile_stride = tb;
+    P.b_lbo = ct * 4;                                   // a column shift = one pixel = 128 bytes
+    P.b_sub_bytes = (32 / g.q) * wt * ct * 4;
+    P.ksteps = ci * bp * g.q / 8;
+    P.chunks = ci > 1 ? (g.n + ci - 1) / ci : g.n * (g.p / bp);
+    P.stages = 200 * 1024 / P.stage_bytes;
+    if (P.stages > kMaxStages) P.stages = kMaxStages;
+    if (P.stages < 2) return false;
+    const int cols = (P.m == 128 ? 2 : 1) * g.s * ct;   // two accumulators: side by side (M = 128) or in the lane halves (M = 64)
+    if ((g.s * ct) % (P.m == 128 ? 16 : 8) != 0) return false;
+    P.tmem_cols = pow2_ceil(cols);
+    if (P.tmem_cols > 512) return false;
+    // instruction descriptor: fp32 accumulate, tf32 x tf32, A K-major, B MN-major, N, M
+    P.idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) | ((uint32_t)(g.s * ct >> 3) << 17) | ((uint32_t)(P.m >> 4) << 24);
+    const int tiles = P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1);
+    if (!choose_splits(P, g, tiles)) return false;
+    if ((size_t)P.m * (g.s * ct + 4) * 4 > 212 * 1024) return false;
+    P.slot_quads = P.m * (g.s * ct / 4);
+    P.qpr_magic = (uint32_t)(((1ull << 32) + (g.s * ct / 4) - 1) / (g.s * ct / 4));
+    P.timeline = env_int("GACONV_TC_TIMELINE", 0);
+#ifdef GACONV_TUNING
+    if (env_int("GACONV_TC_VERBOSE", 0))
+        fprintf(stderr, "plan_tc_f32 c%d k%d pq%d passes%d: m%d ci%d bp%d ksteps%d stage %d B x%d, tiles %d splits %d cl %d chunks %d\n",
+                g.c, g.k, pq, passes, P.m, ci, bp, P.ksteps, P.stage_bytes, P.stages, tiles, P.splits, P.cl, P.chunks);
+#endif
+    out->partial_bytes = P.splits / P.cl > 1 ? (size_t)tiles * (P.splits / P.cl) * P.slot_quads * 16 : 0;
+    // the two planes of each operand, [plane][elements]
+    out->scratch_bytes = passes == 3 ? 2 * ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 4 : 0;
+    out->reads_transposed_dy = false;
+    memcpy(out->opaque, &P, sizeof(P));
+    return encode_fn() != nullptr;
+}
+
 cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, void* scratch, uint32_t* counters,
                       uint32_t* status, const TcPlan& plan, cudaStream_t stream)
 {
@@ -817,7 +967,33 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     if (enc == nullptr) return cudaErrorNotSupported;
 
     CUtensorMap map_dy, map_x;
-    if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) -- (k, n, pq) for the (pixel, image) ordering -- with 64-channel boxes
+    if (P.f32) {
+        const size_t nx = (size_t)g.n * g.c * g.h * g.w, ndy = (size_t)g.n * g.k * pq;
+        const void* xs = x; const void* dys = dy;
+        if (P.passes == 3) {      // planes [big | small] of X, then of dY, in the scratch
+            float* xp = static_cast<float*>(scratch); float* dyp = xp + 2 * nx;
+            const unsigned blocks = 148 * 8;
+            if (launch_kernel(split_tf32_kernel, dim3(blocks), dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float4*>(x),
+                              reinterpret_cast<float4*>(xp), reinterpret_cast<float4*>(xp + nx), nx / 4) != cudaSuccess ||
+                launch_kernel(split_tf32_kernel, dim3(blocks), dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float4*>(dy),
+                              reinterpret_cast<float4*>(dyp), reinterpret_cast<float4*>(dyp + ndy), ndy / 4) != cudaSuccess)
+                return cudaErrorLaunchFailure;
+            note_launch(2);
+            xs = xp; dys = dyp;
+        }
+        const cuuint64_t planes = P.passes == 3 ? 2 : 1;
+        cuuint64_t d4[4] = {(cuuint64_t)pq, (cuuint64_t)g.k, (cuuint64_t)g.n, planes};
+        cuuint64_t s4[3] = {(cuuint64_t)pq * 4, (cuuint64_t)g.k * pq * 4, (cuuint64_t)ndy * 4};
+        cuuint32_t b4[4] = {32, (cuuint32_t)P.kb, 1, 1}, e4[4] = {1, 1, 1, 1};
+        cuuint64_t d5[5] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n, planes};
+        cuuint64_t s5[4] = {(cuuint64_t)g.c * 4, (cuuint64_t)g.w * g.c * 4, (cuuint64_t)g.h * g.w * g.c * 4, (cuuint64_t)nx * 4};
+        cuuint32_t b5[5] = {(cuuint32_t)P.ct, (cuuint32_t)(g.q + g.s - 1), (cuuint32_t)P.bp, (cuuint32_t)P.ci, 1}, e5[5] = {1, 1, 1, 1, 1};
+        if (enc(&map_dy, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(dys), d4, s4, b4, e4, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<void*>(xs), d5, s5, b5, e5, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    } else if (P.tiny) {   // transposed copy dYt[n][pq][k], then a map over (k, pq, n) -- (k, n, pq) for the (pixel, image) ordering -- with 64-channel boxes
         if (dy != nullptr) {
             if (launch_kernel(transpose_dy_kernel, dim3((unsigned)(g.n * ((g.k + 63) / 64))), dim3(128), 0, stream, dim3(1, 1, 1),
                               static_cast<const __nv_bfloat16*>(dy), static_cast<__nv_bfloat16*>(scratch), g.k, pq) != cudaSuccess)
@@ -845,7 +1021,7 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(P.a_sub_px * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
-    {   // X as (c, w, h, n), bf16; a box is ct channels x q columns x rows x ci images, stepping by the conv stride
+    if (!P.f32) {   // X as (c, w, h, n), bf16; a box is ct channels x q columns x rows x ci images, stepping by the conv stride
         cuuint64_t dims[4] = {(cuuint64_t)g.c, (cuuint64_t)g.w, (cuuint64_t)g.h, (cuuint64_t)g.n};
         cuuint64_t strides[3] = {(cuuint64_t)g.c * 2, (cuuint64_t)g.w * g.c * 2, (cuuint64_t)g.h * g.w * g.c * 2};
         const int rows = (P.halo || P.wide) ? P.bp + P.rc - 1 : P.bp;
@@ -869,7 +1045,7 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
     if (red_bytes > smem) smem = red_bytes;
     smem += 1024 + (size_t)P.m * 128;
     dim3 grid(P.tiles_k * P.tiles_c * (P.rsplit ? g.r : 1), P.splits);
-    const int ks = P.a_sub_px / 16;
+    const int ks = P.a_sub_px / (P.f32 ? 8 : 16);
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
     cudaError_t err = cudaErrorInvalidValue;
