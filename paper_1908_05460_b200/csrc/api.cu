@@ -86,13 +86,13 @@ Top1Layout top1_layout(const Geom& g)
 struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; StemPlan sp; bool tc_ok, stem_ok; };
 // fp32 inputs take the tcgen05 kernel (TF32 MMAs on split operands) where the layer is wide enough for the
 // tensor cores to pay for the extra pass that splits the operands; the one-pass TF32 mode needs no split
-bool tc_f32_wanted(const Geom& g, int math) { return !g.bf16 && (math == GACONV_MATH_TF32 || g.c >= 64); }
+bool tc_f32_wanted(const Geom& g, int math, int algo) { return !g.bf16 && (math == GACONV_MATH_TF32 || algo == GACONV_ALGO_TENSOR || g.c >= 64); }
 
-ExactLayout exact_layout(const Geom& g, int math)
+ExactLayout exact_layout(const Geom& g, int math, int algo)
 {
     ExactLayout L;
     L.dp = plan_direct(g);
-    L.tc_ok = g.bf16 ? plan_tc(g, &L.tp) : (tc_f32_wanted(g, math) && plan_tc_f32(g, math == GACONV_MATH_TF32 ? 1 : 3, &L.tp));
+    L.tc_ok = g.bf16 ? plan_tc(g, &L.tp) : (tc_f32_wanted(g, math, algo) && plan_tc_f32(g, math == GACONV_MATH_TF32 ? 1 : 3, &L.tp));
     L.partial_off = kWsDataOffset;
     size_t partial = L.dp.partial_bytes;
     if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
@@ -175,7 +175,7 @@ gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t me
     gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
     switch (method) {
-        case GACONV_METHOD_EXACT: *bytes = exact_layout(g, desc->math).total; return GACONV_OK;
+        case GACONV_METHOD_EXACT: *bytes = exact_layout(g, desc->math, desc->algo).total; return GACONV_OK;
         case GACONV_METHOD_TOP1: *bytes = top1_layout(g).total; return GACONV_OK;
         case GACONV_METHOD_TOPK: {
             const int t = topk_of(desc, g);
@@ -206,7 +206,7 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
-    const ExactLayout L = exact_layout(g, desc->math);
+    const ExactLayout L = exact_layout(g, desc->math, desc->algo);
     const bool mma_ok = direct_mma_supported(g, L.dp);
     if (desc->math == GACONV_MATH_TF32 && !mma_ok && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
     if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
@@ -339,7 +339,7 @@ gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const vo
         st = check_ws(desc, need);
         if (st != GACONV_OK) return st;
         if (method == GACONV_METHOD_EXACT) {
-            const ExactLayout L = exact_layout(g, desc->math);
+            const ExactLayout L = exact_layout(g, desc->math, desc->algo);
             if (desc->math == GACONV_MATH_TF32 && !direct_mma_supported(g, L.dp) && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
             if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
         }

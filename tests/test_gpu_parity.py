@@ -335,6 +335,37 @@ def test_fp32_exact_split_tf32_and_fp32_pipes(li):
     assert B.gaconv_poll_async_status(auto.desc) == B.OK
 
 
+# ---- fp32 inputs on the tcgen05 kernel (kind::tf32), forced: three passes on split operands, and one plain TF32 pass ----
+TC_F32_SHAPES = [
+    ConvLayer("tcf32 64->64@8 M64", 9, 64, 8, 8, 64, 3, 3, 1, 1),
+    ConvLayer("tcf32 64->128@16 M128", 5, 64, 16, 16, 128, 3, 3, 1, 1),
+    ConvLayer("tcf32 96->72@8 ragged k, three c tiles", 7, 96, 8, 8, 72, 3, 3, 1, 1),
+    ConvLayer("tcf32 32->200@16 two k tiles, ragged", 3, 32, 16, 16, 200, 3, 3, 1, 1),
+    ConvLayer("tcf32 32->32@32 rows of 32", 4, 32, 32, 32, 32, 3, 3, 1, 1),
+    ConvLayer("tcf32 1x1 64->48@16", 6, 64, 16, 16, 48, 1, 1, 1, 0),
+    ConvLayer("tcf32 5x5 64->64@16", 3, 64, 16, 16, 64, 5, 5, 1, 2),
+    ConvLayer("tcf32 7x7 32->16@8", 4, 32, 8, 8, 16, 7, 7, 1, 3),
+    ConvLayer("tcf32 many images", 200, 32, 8, 8, 32, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("li", range(len(TC_F32_SHAPES)), ids=[l.name for l in TC_F32_SHAPES])
+def test_fp32_on_tcgen05_matches_oracle(li):
+    layer = TC_F32_SHAPES[li]
+    x, dy = _inputs(layer, torch.float32, 340 + li)
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.5)
+    g = GpuLayer(layer, torch.float32, x, dy, alpha=0.5, algo=B.ALGO_TENSOR)
+    got = g.exact()
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+    assert norm_err(got, ref, dn) <= TOL_F32                     # big*big + big*small + small*big, fp32 accumulation
+    np.testing.assert_array_equal(got, g.exact())
+    one = GpuLayer(layer, torch.float32, x, dy, alpha=0.5, algo=B.ALGO_TENSOR, math=B.MATH_TF32)
+    e1 = norm_err(one.exact(), ref, dn)
+    assert TOL_F32 < e1 <= 4e-3                                   # one pass really is TF32: outside the fp32 class, inside its own
+    kcrs = GpuLayer(layer, torch.float32, x, dy, alpha=0.5, algo=B.ALGO_TENSOR, dw_layout=B.DW_KCRS)
+    np.testing.assert_array_equal(kcrs.exact(), got)
+
+
 def test_tf32_mode_is_refused_where_it_has_no_kernel():
     layer = ConvLayer("7x7", 2, 16, 16, 16, 16, 7, 7, 1, 3)
     x, dy = _inputs(layer, torch.float32, 320)
