@@ -622,20 +622,25 @@ reduce_slots_kernel(const float4* __restrict__ partial, float* __restrict__ dw, 
 // fp32 operand -> two planes: big = x with the 13 low mantissa bits cleared (exactly a TF32 number) and
 // small = x - big (exact in fp32; at most 13 significant bits, of which the tensor core keeps 11).  Then
 // a*b = big_a*big_b + big_a*small_b + small_a*big_b up to ~2^-21 |a*b|.
+__device__ __forceinline__ void split4(const float4 v, float4& b, float4& sm)
+{
+    b.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); sm.x = v.x - b.x;
+    b.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); sm.y = v.y - b.y;
+    b.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); sm.z = v.z - b.z;
+    b.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); sm.w = v.w - b.w;
+}
+// one launch for both operands: vectors [0, nx) are X's, [nx, nx + ndy) dY's; planes [big | small] of each
 __global__ void __launch_bounds__(256)
-split_tf32_kernel(const float4* __restrict__ src, float4* __restrict__ big, float4* __restrict__ small, size_t nvec)
+split_tf32_kernel(const float4* __restrict__ x, float4* __restrict__ xp, size_t nx,
+                  const float4* __restrict__ dy, float4* __restrict__ dyp, size_t ndy)
 {
     pdl_release_next_grid();
     pdl_wait_prior_grid();
     const size_t stride = (size_t)gridDim.x * blockDim.x;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        const float4 v = __ldg(src + i);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nx + ndy; i += stride) {
         float4 b, sm;
-        b.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u); sm.x = v.x - b.x;
-        b.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u); sm.y = v.y - b.y;
-        b.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u); sm.z = v.z - b.z;
-        b.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u); sm.w = v.w - b.w;
-        big[i] = b; small[i] = sm;
+        if (i < nx) { split4(__ldg(x + i), b, sm); xp[i] = b; xp[nx + i] = sm; }
+        else { const size_t j = i - nx; split4(__ldg(dy + j), b, sm); dyp[j] = b; dyp[ndy + j] = sm; }
     }
 }
 
@@ -709,19 +714,28 @@ bool choose_splits(TcParams& P, const Geom& g, int tiles)
     // Measured on the layer shapes of the three networks: a cluster whose splits cover the whole tile (no workspace,
     // no second kernel) wins even at two thirds of the CTAs; otherwise the largest cluster that keeps 85% of them.
     const int cl_force = env_int("GACONV_TC_FORCE_CL", 0);
-    int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0}, most = 0;
+    int sp_of[5] = {0, 0, 0, 0, 0}, per_of[5] = {0, 0, 0, 0, 0};
+    bool fits[5] = {false, false, false, false, false};      // the whole grid is resident at once (no second wave)
     for (int c = 1; c <= 4; ++c) {
         if (c > cl_cap || c > max_splits || (cl_force && c != cl_force)) continue;
         // clusters per tile: within the split budget and, where the tiles allow it, within one resident wave
-        per_of[c] = std::min(max_splits / c, std::max(1, std::min(resident_clusters(c), std::max(1, sms / c)) / tiles));
+        const int wave = std::min(resident_clusters(c), std::max(1, sms / c));
+        per_of[c] = std::min(max_splits / c, std::max(1, wave / tiles));
         sp_of[c] = per_of[c] * c;
-        most = std::max(most, sp_of[c]);
+        fits[c] = tiles * per_of[c] <= wave;
     }
+    // a cluster size whose grid needs a second wave (a few clusters left over that run alone) is taken only if
+    // every size does
+    bool any_fit = false;
+    for (int c = 1; c <= 4; ++c) any_fit = any_fit || (sp_of[c] > 0 && fits[c]);
+    int most = 0;
+    for (int c = 1; c <= 4; ++c)
+        if (sp_of[c] > 0 && (fits[c] || !any_fit)) most = std::max(most, sp_of[c]);
     int cl = 0, splits = 0;
     for (int c = 4; c >= 1 && cl == 0; --c)
-        if (per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
+        if ((fits[c] || !any_fit) && per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
     for (int c = 4; c >= 1 && cl == 0; --c)
-        if (sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
+        if ((fits[c] || !any_fit) && sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
     if (cl == 0) return false;
     P.cl = cl;
     P.splits = splits;
@@ -974,11 +988,9 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
             float* xp = static_cast<float*>(scratch); float* dyp = xp + 2 * nx;
             const unsigned blocks = 148 * 8;
             if (launch_kernel(split_tf32_kernel, dim3(blocks), dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float4*>(x),
-                              reinterpret_cast<float4*>(xp), reinterpret_cast<float4*>(xp + nx), nx / 4) != cudaSuccess ||
-                launch_kernel(split_tf32_kernel, dim3(blocks), dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float4*>(dy),
-                              reinterpret_cast<float4*>(dyp), reinterpret_cast<float4*>(dyp + ndy), ndy / 4) != cudaSuccess)
+                              reinterpret_cast<float4*>(xp), nx / 4, static_cast<const float4*>(dy), reinterpret_cast<float4*>(dyp), ndy / 4) != cudaSuccess)
                 return cudaErrorLaunchFailure;
-            note_launch(2);
+            note_launch();
             xs = xp; dys = dyp;
         }
         const cuuint64_t planes = P.passes == 3 ? 2 : 1;
