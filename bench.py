@@ -283,8 +283,26 @@ def run_one_layer(args):
         ee.record()
         ee.synchronize()
         ts.append(es.elapsed_time(ee) * 1e3 / copies)
+    launches = B.gaconv_launch_count()
+    # the same burst replayed from a CUDA graph: launch cost off the host, as inside a captured training step
+    graph_us = None
+    if not args.no_graph:
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            for xb, dyb in bufs:
+                one(xb, dyb)
+        gr.replay()
+        torch.cuda.synchronize()
+        tg = []
+        for _ in range(max(1, args.layer_iters)):
+            es.record()
+            gr.replay()
+            ee.record()
+            ee.synchronize()
+            tg.append(es.elapsed_time(ee) * 1e3 / copies)
+        graph_us = statistics.median(tg)
     print(json.dumps({"layer": args.layer, "dtype": dname, "method": args.method, "us_per_call_host_launched": statistics.median(ts),
-                      "copies": copies, "status": B.gaconv_poll_async_status(desc), "launches": B.gaconv_launch_count()}))
+                      "us_per_call_graph": graph_us, "copies": copies, "status": B.gaconv_poll_async_status(desc), "launches": launches}))
     del ws
 
 

@@ -31,22 +31,26 @@ __device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint
     c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
 }
 
+// Box-Muller on the special-function unit.  The result has to be within 1e-5 * max(1, |z|) of the real-number
+// value of the formula, which leaves room for the fast approximations as long as no argument is rounded where
+// rounding is amplified:
+//   ln u1   u1 = (wa+1) 2^-32.  Away from 1 the hardware logarithm of the rounded value is accurate to ~2^-21
+//           in absolute terms; for u1 > 1 - 2^-7 the logarithm is small and that is not enough, but there
+//           1-u1 = t 2^-32 with t an integer below 2^25 (exact in fp32 up to rounding of 2^-24 relative) and
+//           ln(1-f) = -(f + f^2/2 + f^3/3 + f^4/4) is accurate to f^5/5 < 2^-37.
+//   angle   2 pi u2 with u2 = wb 2^-32: taking wb as a signed integer moves the angle to [-pi, pi), where the
+//           hardware sine and cosine have their stated absolute accuracy (2^-21.4), without changing the value.
 __device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float& z0, float& z1)
 {
-    // ln u1 with u1 = (wa+1) 2^-32, in fp32 without losing u1 near 1: below one half take the
-    // logarithm of the (rounded) value itself -- a relative error of 2^-24 in u1 is an absolute error
-    // of 2^-24 in ln u1; above, 1-u1 = t 2^-32 with t an integer, and log1p keeps its relative accuracy.
-    float ln_u1;
-    if (wa < 0x7fffffffu) {
-        ln_u1 = logf((float)(wa + 1u) * (1.0f / 4294967296.0f));
-    } else {
-        const uint32_t t = 0xffffffffu - wa;                 // 2^32 - (wa+1)
-        ln_u1 = log1pf(-(float)t * (1.0f / 4294967296.0f));
-    }
-    const float rho = sqrtf(-2.0f * ln_u1);
-    float sn, cs;
-    sincospif(2.0f * ((float)wb * (1.0f / 4294967296.0f)), &sn, &cs);
-    z0 = rho * cs; z1 = rho * sn;
+    const uint32_t t = 0xffffffffu - wa;                          // 2^32 - (wa+1)
+    const float f = (float)t * (1.0f / 4294967296.0f);            // 1 - u1
+    const float u1 = (wa < 0x7fffffffu) ? (float)(wa + 1u) * (1.0f / 4294967296.0f) : 1.0f - f;
+    const float ln_far = __logf(u1);
+    const float ln_near = -f * fmaf(f, fmaf(f, fmaf(f, 0.25f, 1.0f / 3.0f), 0.5f), 1.0f);
+    const float ln_u1 = (t < (1u << 25)) ? ln_near : ln_far;
+    const float rho = __fsqrt_rn(-2.0f * ln_u1);
+    const float theta = (float)(int32_t)wb * (6.283185307179586f / 4294967296.0f);
+    z0 = rho * __cosf(theta); z1 = rho * __sinf(theta);
 }
 
 // philox words of counter j -> four standard normals

@@ -158,6 +158,14 @@ def test_zero_and_random_methods():
     gb = GpuLayer(big, torch.float32, torch.zeros(1, 256, 4, 4), torch.zeros(1, 256, 4, 4), dw_layout=B.DW_KCRS)
     v = gb.approx(B.METHOD_RANDOM, seed=77).reshape(-1) * 128
     assert abs(v.mean()) < 4 / np.sqrt(v.size) and abs(v.std() - 1) < 0.01
+    # every value of a large layer (2.4 million draws reach u1 within 1e-6 of 0 and of 1), both storage orders
+    wide = ConvLayer("wide", 1, 512, 4, 4, 512, 3, 3, 1, 1)
+    for layout in (B.DW_KCRS, B.DW_KRSC):
+        gw = GpuLayer(wide, torch.float32, torch.zeros(1, 512, 4, 4), torch.zeros(1, 512, 4, 4), dw_layout=layout, rand_std=1.0)
+        got = gw.approx(B.METHOD_RANDOM, seed=2024).reshape(-1)
+        ref = oracle.dw_random(got.size, 2024, 1.0)
+        assert np.max(np.abs(got - ref) / np.maximum(1.0, np.abs(ref))) <= 1e-5
+        assert np.abs(ref).max() > 4.5 and np.abs(ref).min() < 1e-5          # the sample does reach both tails
 
 
 def test_runs_are_bitwise_reproducible():
