@@ -55,14 +55,14 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     return GACONV_OK;
 }
 
-// Small maps with many channels: the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes) cost more
-// than the dense contraction on tensor cores, and with few pixels per map the sparse tensor is not
-// that sparse (1 - 1/(PQ), Section 2.3).  Then the method is run literally as the paper states it:
-// build the sparse version of dY (one entry per map, the signed sum) and take its exact filter
-// gradient with the tensor-core kernel.
+// Maps of at most 4x4 pixels with many channels: the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes,
+// the same number of bytes gathered from L2) cost more than the dense contraction on tensor cores, and with so few
+// pixels per map the sparse tensor is not that sparse (1 - 1/(PQ), Section 2.3).  Then the method is run
+// literally as the paper states it: build the sparse version of dY (one entry per map, the signed sum) and take
+// its exact filter gradient with the tensor-core kernel.  (On 8x8 maps the gather kernel measured faster.)
 bool top1_dense_route(const Geom& g, TcPlan* tp)
 {
-    return g.bf16 && g.p * g.q <= 64 && g.c >= 128 && plan_tc(g, tp);
+    return g.bf16 && g.p * g.q <= 16 && g.c >= 128 && plan_tc(g, tp);
 }
 
 struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, scratch_off, total; GatherPlan gp; TcPlan tp; bool dense; };

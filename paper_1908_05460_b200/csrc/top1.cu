@@ -229,6 +229,15 @@ __device__ __forceinline__ Raw4 ld4_raw(const __nv_bfloat16* p) {
     const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
     return Raw4{{t.x, t.y, 0u, 0u}};
 }
+__device__ __forceinline__ Raw4 ld8_raw(const __nv_bfloat16* p) {          // eight channels
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    return Raw4{{t.x, t.y, t.z, t.w}};
+}
+__device__ __forceinline__ Raw4 ld8_raw(const float* p) { return ld4_raw(p); }   // (never used: fp32 loads are 16 bytes already)
+__device__ __forceinline__ void raw_to_float8(const Raw4& r, float (&v)[8]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(r.w[i] << 16); v[2 * i + 1] = __uint_as_float(r.w[i] & 0xffff0000u); }
+}
 __device__ __forceinline__ void raw_to_float(const Raw4& r, const float*, float (&v)[4]) {
     v[0] = __uint_as_float(r.w[0]); v[1] = __uint_as_float(r.w[1]); v[2] = __uint_as_float(r.w[2]); v[3] = __uint_as_float(r.w[3]);
 }
@@ -244,7 +253,7 @@ __device__ __forceinline__ void raw_to_float(const Raw4& r, const __nv_bfloat16*
 //   phase 3  after a cluster barrier, CTA j adds slice j of the block over the CL CTAs through
 //            distributed shared memory, in rank order, and writes alpha * total to dW.
 // No global scratch, no atomics; the order of every sum is fixed.
-template <typename T, bool VEC>
+template <typename T, bool VEC, bool WIDE>
 __global__ void __launch_bounds__(512, 2)
 top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x, int NJ)
 {
@@ -254,11 +263,10 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int rsc = g.r * g.s * g.c;
     float* s_part = reinterpret_cast<float*>(smem_raw);                 // [rsc]
-    int* s_h0 = reinterpret_cast<int*>(s_part + rsc);                   // [ipc] top-left input row of each patch
-    int* s_w0 = s_h0 + ipc;
-    float* s_sum = reinterpret_cast<float*>(s_w0 + ipc);
-    long long* s_base = reinterpret_cast<long long*>(smem_raw + (((size_t)rsc * 4 + (size_t)ipc * 12 + 7) & ~(size_t)7));   // [ipc] element offset of each patch's top-left pixel
-    float* s_subs = reinterpret_cast<float*>(s_base + ipc);            // [NJ][rsc] lane subtotals
+    // per image of this CTA, one 16-byte record: {element offset of the patch's top-left pixel (64 bits), the signed
+    // sum (float bits), validity bits: bit r = patch row r lies inside the image, bit 16+s = patch column s does}
+    uint4* s_rec = reinterpret_cast<uint4*>(smem_raw + (((size_t)rsc * 4 + 15) & ~(size_t)15));      // [ipc]
+    float* s_subs = reinterpret_cast<float*>(s_rec + ipc);              // [NJ][rsc] lane subtotals
 
     const int k = blockIdx.y, chunk = blockIdx.x, CL = gridDim.x;
     const int n0 = chunk * ipc;
@@ -276,9 +284,11 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
             scan_map<T, VEC>(dy + ((long long)(n0 + (live ? i : 0)) * g.k + k) * pq, live, pq, G, sub, best_j, s);
             if (live && sub == 0) {
                 const int h0 = (best_j / g.q) * g.stride_h - g.pad_h, w0 = (best_j % g.q) * g.stride_w - g.pad_w;
-                s_h0[i] = h0; s_w0[i] = w0;
-                s_base[i] = (long long)i * g.xs_n + (long long)h0 * g.xs_h + (long long)w0 * g.xs_w;
-                s_sum[i] = s;
+                const long long base = (long long)i * g.xs_n + (long long)h0 * g.xs_h + (long long)w0 * g.xs_w;
+                uint32_t mask = 0;
+                for (int r = 0; r < g.r; ++r) mask |= (uint32_t)((unsigned)(h0 + r) < (unsigned)g.h) << r;
+                for (int c = 0; c < g.s; ++c) mask |= (uint32_t)((unsigned)(w0 + c) < (unsigned)g.w) << (16 + c);
+                s_rec[i] = make_uint4((uint32_t)(unsigned long long)base, (uint32_t)((unsigned long long)base >> 32), __float_as_uint(s), mask);
             }
         }
     }
@@ -291,44 +301,63 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
     // the NJ subtotals are then added in lane order.  VX elements per group: four channels per load
     // on the vector path (NHWC, C a multiple of four), else one.
     {
-        const int VX = vec_x ? 4 : 1;
-        constexpr int BATCH = sizeof(T) == 4 ? 4 : 8;          // loads in flight per thread (register budget: 64)
+        // WIDE (bf16, C a multiple of eight): eight channels per 16-byte load, four loads in flight
+        const int VX = WIDE ? 8 : vec_x ? 4 : 1;
+        constexpr int BATCH = (sizeof(T) == 4 || WIDE) ? 4 : 8;          // loads in flight per thread (register budget: 64)
+        constexpr int NV = WIDE ? 8 : 4;
         const int groups = rsc / VX;
         float* s_sub = NJ > 1 ? s_subs : s_part;               // NJ == 1: results go straight to s_part
         for (int item = threadIdx.x; item < groups * NJ; item += blockDim.x) {
             const int j = item / groups, e = (item - j * groups) * VX;
             const int c = e % g.c, rs = e / g.c, s = rs % g.s, r = rs / g.s;
             const T* xc = x + n0 * g.xs_n + c * g.xs_c + r * g.xs_h + s * g.xs_w;     // this element of a patch whose corner is pixel (0,0)
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t bits = (1u << r) | (1u << (16 + s));
+            float acc[NV];
+#pragma unroll
+            for (int t = 0; t < NV; ++t) acc[t] = 0.f;
             for (int i0 = j; i0 < cnt; i0 += BATCH * NJ) {
                 // BATCH loads are issued before any is consumed; they stay raw (two or four registers each)
-                // until then, so that the register allocator has no reason to serialise them
+                // until then, so that the register allocator has no reason to serialise them.  A patch element
+                // outside the image contributes weight 0 times a zero that is not loaded.
                 Raw4 raw[BATCH];
-                float one[BATCH];
-                bool okv[BATCH];
+                float wsum[BATCH];
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
                     const int i = i0 + u * NJ;
                     const bool in = i < cnt;
-                    okv[u] = in && (unsigned)(s_h0[in ? i : 0] + r) < (unsigned)g.h && (unsigned)(s_w0[in ? i : 0] + s) < (unsigned)g.w;
-                    const T* p = okv[u] ? xc + s_base[i] : x;                           // element 0 is always readable
-                    if (vec_x) raw[u] = ld4_raw(p);
-                    else one[u] = ldf(p);
+                    const uint4 rec = s_rec[in ? i : 0];
+                    const bool ok = in && (rec.w & bits) == bits;
+                    wsum[u] = ok ? __uint_as_float(rec.z) : 0.f;
+                    const T* p = xc + (long long)(((unsigned long long)rec.y << 32) | rec.x);
+                    raw[u] = Raw4{{0u, 0u, 0u, 0u}};
+                    if (ok) {
+                        if (WIDE) raw[u] = ld8_raw(p);
+                        else if (vec_x) raw[u] = ld4_raw(p);
+                        else raw[u].w[0] = __float_as_uint(ldf(p));
+                    }
                 }
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
-                    const int i = i0 + u * NJ;
-                    if (i < cnt && okv[u]) {
-                        const float sm_ = s_sum[i];
-                        float v[4];
-                        if (vec_x) raw_to_float(raw[u], static_cast<const T*>(nullptr), v);
-                        else { v[0] = one[u]; v[1] = v[2] = v[3] = 0.f; }
+                    float v[NV];
+                    if constexpr (WIDE) raw_to_float8(raw[u], v);
+                    else {
+                        float v4[4];
+                        if (vec_x) raw_to_float(raw[u], static_cast<const T*>(nullptr), v4);
+                        else { v4[0] = __uint_as_float(raw[u].w[0]); v4[1] = v4[2] = v4[3] = 0.f; }
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) acc[t] = fmaf(sm_, v[t], acc[t]);
+                        for (int t = 0; t < 4; ++t) v[t] = v4[t];
                     }
+#pragma unroll
+                    for (int t = 0; t < NV; ++t) acc[t] = fmaf(wsum[u], v[t], acc[t]);
                 }
             }
-            for (int t = 0; t < VX; ++t) s_sub[j * rsc + e + t] = acc[t];
+            float* out = s_sub + j * rsc + e;
+            if (VX >= 4) {            // 16-byte stores: rsc and e are multiples of four here
+                *reinterpret_cast<float4*>(out) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                if constexpr (WIDE) *reinterpret_cast<float4*>(out + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            } else {
+                out[0] = acc[0];
+            }
         }
         if (NJ > 1) {
             __syncthreads();
@@ -511,10 +540,10 @@ cudaError_t launch_gather(const void* x, const int32_t* idx, const float* sum, f
 bool top1_fused_supported(const Geom& g)
 {
     // the per-channel block of R*S*C sums lives in shared memory
-    return (size_t)g.r * g.s * g.c * sizeof(float) <= 100 * 1024 && g.k <= 65535;
+    return (size_t)g.r * g.s * g.c * sizeof(float) <= 100 * 1024 && g.k <= 65535 && g.r <= 16 && g.s <= 16;
 }
 
-template <typename T, bool VEC>
+template <typename T, bool VEC, bool WIDE>
 static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom& g, int cl, int ipc, int G, cudaStream_t stream)
 {
     // block of sums + per-image arrays + up to 16 lane subtotals when the block is small
@@ -524,20 +553,23 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     // 512 threads (two CTAs per SM) where the grid still fits in one wave and the scan would otherwise need
     // two passes over the CTA's maps; measured: helps 32-channel layers, neutral or worse for 16 and 64
     const int threads = (g.k >= 32 && (long long)cl * g.k <= 148 * 2) ? 512 : 256;
-    const int groups = rsc / (vec_x ? 4 : 1);
-    const int batch = sizeof(T) == 4 ? 4 : 8;
-    while (nj < 16 && (nj * batch < ipc || nj * 2 * groups <= threads)) nj *= 2;    // one batch of images per lane, no idle threads
+    const int groups = rsc / (WIDE ? 8 : vec_x ? 4 : 1);
+    const int batch = (sizeof(T) == 4 || WIDE) ? 4 : 8;
+    (void)batch;
+    while (nj < 16 && nj * 2 <= ipc && nj * 2 * groups <= threads) nj *= 2;        // image lanes: as many as keep every item on its own thread
     while (nj > 1 && (size_t)rsc * 4 * (1 + nj) > 150 * 1024) nj /= 2;              // the subtotals must fit shared memory
-    const size_t smem = (((size_t)rsc * 4 + (size_t)ipc * 12 + 7) & ~(size_t)7) + (size_t)ipc * 8 + (nj > 1 ? (size_t)nj * rsc * 4 : 0) + 16;
-    static size_t configured = 0;
-    if (smem > 48 * 1024 && smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(top1_fused_kernel<T, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = (((size_t)rsc * 4 + 15) & ~(size_t)15) + (size_t)ipc * 16 + (nj > 1 ? (size_t)nj * rsc * 4 : 0) + 16;
+    static size_t configured[64] = {};           // per device: the attribute belongs to the device's copy of the kernel
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (smem > 48 * 1024 && smem > configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(top1_fused_kernel<T, VEC, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = smem;
+        configured[dev] = smem;
     }
     // lanes per map: few enough that one pass covers all the CTA's maps (their loads are then all in flight at once)
     while (G > 1 && G * ipc > threads) G /= 2;
-    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj);
+    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC, WIDE>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj);
     note_launch();
     return e;
 }
@@ -553,12 +585,15 @@ cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Ge
     const MapScanShape m = map_scan_shape(g);
     if (g.bf16) {
         auto xx = static_cast<const __nv_bfloat16*>(x); auto dd = static_cast<const __nv_bfloat16*>(dy);
-        return m.vec ? launch_fused_t<__nv_bfloat16, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
-                     : launch_fused_t<__nv_bfloat16, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
+        const bool wide = g.xs_c == 1 && g.c % 8 == 0 && g.xs_w % 8 == 0;     // 16-byte aligned groups of eight channels
+        if (wide) return m.vec ? launch_fused_t<__nv_bfloat16, true, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
+                               : launch_fused_t<__nv_bfloat16, false, true>(xx, dd, dw, g, cl, ipc, m.G, stream);
+        return m.vec ? launch_fused_t<__nv_bfloat16, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream)
+                     : launch_fused_t<__nv_bfloat16, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
     }
     auto xx = static_cast<const float*>(x); auto dd = static_cast<const float*>(dy);
-    return m.vec ? launch_fused_t<float, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
-                 : launch_fused_t<float, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
+    return m.vec ? launch_fused_t<float, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream)
+                 : launch_fused_t<float, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
 }
 
 }  // namespace gaconv
