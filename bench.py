@@ -183,6 +183,16 @@ def run_reference(args, layers):
 
 
 # ------------------------------------------------------------------------------------------------
+def layer_sm_budget(layer, eb, peaks, args):
+    """SMs a layer is sized for when the layers of a step run next to one another on several lanes: a share that
+    grows with the layer's roofline time (the minimum for the latency-bound layers, up to the maximum)."""
+    if args.lanes == 1:
+        return 0
+    t_roof = max(layer.flops_exact() / (peaks["bf16_tflops"] * 1e12 * (1.0 if eb == 2 else 0.5)),
+                 layer.bytes_exact(eb) / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    return max(args.budget_min, min(args.budget_max, int(148 * t_roof / args.budget_div)))
+
+
 def run_sweep(args):
     """Approximation-schedule sweep: ResNet-20 and VGG-19 layer sets at batch 256, bf16.  A seeded mask
     approximates a fraction f of the layers (top-1 method) on odd steps; even steps are all exact.
@@ -195,6 +205,7 @@ def run_sweep(args):
     build_mod.build()
     B.load()
     torch.cuda.set_device(0)
+    peaks = measured_peaks()
     out = {"workload": "schedule sweep, N=%d, bf16, seeded mask on odd steps, top-1 method, %d lanes" % (args.sweep_batch, args.lanes), "nets": {}}
     es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for cfg, name in ((2, "resnet20"), (4, "vgg19")):
@@ -203,7 +214,7 @@ def run_sweep(args):
         slots = []
         for li, l in enumerate(layers):
             x, dy = I.make_layer_inputs(l, torch.bfloat16, 5, li + 100 * cfg)
-            d = B.make_desc(l, torch.bfloat16, alpha=1.0 / l.n)
+            d = B.make_desc(l, torch.bfloat16, alpha=1.0 / l.n, sm_budget=layer_sm_budget(l, 2, peaks, args))
             slots.append((I.to_nhwc(x).cuda(), dy.cuda(),
                           torch.empty(l.k, l.r, l.s, l.c, dtype=torch.float32, device="cuda"), d, B.attach_workspace(d)))
         rows = []
@@ -387,9 +398,7 @@ def main():
                 s.ws = B.attach_workspace(s.desc)
                 # the step runs layers next to one another on several lanes: each layer is sized for a share of the SMs
                 # that grows with its roofline time (18 SMs for the latency-bound layers, up to half the GPU)
-                t_roof = max(l.flops_exact() / (peaks["bf16_tflops"] * 1e12 * (1.0 if s.eb == 2 else 0.5)),
-                             l.bytes_exact(s.eb) / (peaks["hbm_gbs"] * 1e9)) * 1e6
-                s.budget = 0 if args.lanes == 1 else max(args.budget_min, min(args.budget_max, int(148 * t_roof / args.budget_div)))
+                s.budget = layer_sm_budget(l, s.eb, peaks, args)
                 s.step_desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n, sm_budget=s.budget)
                 s.step_ws = B.attach_workspace(s.step_desc)
                 h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs

@@ -59,7 +59,7 @@ typedef enum {
 /* kernel family; AUTO picks the fastest that supports the shape */
 typedef enum { GACONV_ALGO_AUTO = 0, GACONV_ALGO_DIRECT = 1, GACONV_ALGO_TENSOR = 2 } gaconv_algo_t;
 
-/* Problem statement of one layer (Section 2.4: "input tensor I and output gradient tensor dO"). */
+/* Problem statement of one layer (Section 2.4: the input activations I and the output gradient dO). */
 typedef struct gaconv_conv_desc {
     uint32_t struct_size;              /* = sizeof(gaconv_conv_desc_t); versions the struct               */
     int32_t  n, c, h, w;               /* X is n x c x h x w                                              */
@@ -144,7 +144,7 @@ gaconv_status_t gaconv_poll_async_status_static(void *stream);
  *   GACONV_METHOD_TOP1   (2.3, Algorithm 1)  for every (n,k): keep only the largest-magnitude entry of
  *        dy[n,k,:,:] (lowest p*Q+q among equals), replace it by the signed sum of the map, and take
  *        the exact filter gradient of that sparse tensor.
- *   GACONV_METHOD_TOPK   (2.3: the method "can be modified" to keep the k largest magnitudes, with an
+ *   GACONV_METHOD_TOPK   (2.3 notes that more than one entry per map may be kept, i.e. the k largest magnitudes, with an
  *        adjusted scale that the paper leaves open)  keep the desc->topk largest-magnitude entries of every
  *        map (equal magnitudes: lower p*Q+q first), give each of them sum/topk, and take the exact filter
  *        gradient of that sparse tensor.  topk = 1 is TOP1; topk is clamped to P*Q.
@@ -152,7 +152,7 @@ gaconv_status_t gaconv_poll_async_status_static(void *stream);
 gaconv_status_t gaconv_dw_approx(int32_t method, const void *x, const void *dy, float *dw,
                                  const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
 
-/* Selection step of Algorithm 1 alone ("arg max abs" and "sum" lines), for inspection:
+/* Selection step of Algorithm 1 alone (its arg-max-of-magnitude and sum statements), for inspection:
  *   idx[n*K+k] = p*Q+q of the retained entry, sum[n*K+k] = signed sum of dy[n,k,:,:] (fp32).
  * dy_sparse (may be NULL) receives the dense sparse tensor in dy's dtype and layout: the sum, rounded
  * to in_dtype, at the retained position and zero elsewhere.  Needs no workspace. */

@@ -156,7 +156,15 @@ direct_tiled_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __
             if (!mbar_wait(smem_u32(&bar_full[stage]), phase[stage])) s_fail = 1;   // bounded wait gave up
             phase[stage] ^= 1u;
             __syncthreads();
-            if (s_fail) { if (threadIdx.x == 0) atomicOr(status, 1u); break; }       // uniform exit
+            if (s_fail) {                                                            // uniform exit
+                if (threadIdx.x == 0) {
+                    atomicOr(status, 1u);
+                    // the next item's copies are already in flight: let them land (bounded) before the CTA's memory is released
+                    if (it + 1 < it_end) (void)mbar_wait(smem_u32(&bar_full[stage ^ 1]), phase[stage ^ 1]);
+                }
+                __syncthreads();
+                break;
+            }
         } else {
             __syncthreads();
         }

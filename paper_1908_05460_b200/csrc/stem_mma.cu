@@ -97,7 +97,15 @@ stem_mma_kernel(float* __restrict__ dw, float* __restrict__ partial, uint32_t* _
         if (!mbar_wait(smem_u32(&bar_full[stage]), ph)) s_fail = 1;          // bounded wait gave up
         if (stage) phase1 ^= 1u; else phase0 ^= 1u;
         __syncthreads();
-        if (s_fail) { if (threadIdx.x == 0) atomicOr(status, 1u); break; }   // uniform exit
+        if (s_fail) {                                                        // uniform exit
+            if (threadIdx.x == 0) {
+                atomicOr(status, 1u);
+                // the next item's copies are already in flight: let them land (bounded) before the CTA's memory is released
+                if (it + 1 < it_end) (void)mbar_wait(smem_u32(&bar_full[stage ^ 1]), stage ? phase0 : phase1);
+            }
+            __syncthreads();
+            break;
+        }
         const uint8_t* s_dy = smem + stage * stage_bytes;
         const T* s_x = reinterpret_cast<const T*>(s_dy + dy_bytes);
 

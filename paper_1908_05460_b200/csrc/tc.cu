@@ -22,11 +22,21 @@
 // once a counter shows them complete -- measured slower: the first serialises megabytes of slot reads on
 // a few CTAs, the second needs the whole grid resident, which cluster placement does not guarantee.)
 //
-// Warp roles: warp 0 = TMA producer; warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns
-// the TMEM allocation); warps 4..7 = epilogue.  The filter rows are dealt round-robin to the issuers:
-// a single thread sustains only one small MMA per ~60-100 cycles, and rows accumulate independently.
-// A CTA that holds a single filter row keeps TWO accumulators for it: two issuers take alternate chunks
-// of the reduction, and the epilogue adds accumulator 0 + accumulator 1 (a fixed order).
+// Warp roles: warp 0 = TMA producer (the whole warp: lane b issues copy b of a stage, so the per-copy issue
+// cost overlaps); warps 1..3 = MMA issuers (one elected thread each; warp 1 also owns the TMEM allocation);
+// all eight warps run the epilogue.  The filter rows are dealt round-robin to the issuers: a single thread
+// sustains only one small MMA per ~100 cycles, and rows accumulate independently.  A CTA that holds a single
+// filter row keeps TWO accumulators for it: two issuers take alternate chunks of the reduction, and the
+// epilogue adds accumulator 0 + accumulator 1 (a fixed order).
+//
+// Small maps (at most 16 pixels): both operands are MN-major with 128-byte rows of 64 channels (dY through a
+// transposed copy), the reduction index is ordered (pixel, image) through tensor maps with permuted dimensions,
+// and a chunk's X arrives as one haloed tile, so a filter shift is again a descriptor offset.
+//
+// fp32 inputs: kind::tf32 on operands split into two planes (the upper mantissa bits and the remainder), three
+// MMAs per k-step (big*big + big*small + small*big); an MN-major 32-bit operand uses the 128-byte swizzle on
+// 32-byte units.  One plain TF32 pass on request.
+//
 // Every mbarrier wait is bounded; on expiry the kernel raises the workspace status word, drains
 // the copies it has in flight, frees its tensor memory and returns.
 #include <cuda.h>

@@ -7,7 +7,7 @@ def _layers(kind, L, step, **kw):
 
 
 def test_first_schedule_counts_match_the_paper():
-    # "four approximated layers for VGG-19 and five approximated layers for ResNet-20"
+    # Section 3: the first schedule approximates four layers of VGG-19 and five of ResNet-20
     for step in range(4):
         assert _layers(so.EVERY_4TH_LAYER, 19, step) == [2, 6, 10, 14, 18]
         assert _layers(so.EVERY_4TH_LAYER, 16, step) == [2, 6, 10, 14]
