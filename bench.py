@@ -47,21 +47,21 @@ def workload_sets(config: int, batch: int, dtypes=None):
     return sets
 
 
-def traffic_from_profiles(kernel: str):
-    """DRAM bytes of one captured launch of `kernel`, from the table in profiles/dram_traffic.md (rows:
-    | kernel | layer | dram read B | dram write B | algorithmic B | source |).  None when no row matches."""
+def traffic_from_profiles(kernel: str, family: str):
+    """DRAM bytes of one captured launch of `kernel` on a layer of `family`, from the table in profiles/dram_traffic.md
+    (rows: | kernel | family | layer | dram read B | dram write B | algorithmic B | source |).  None when no row matches."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.md")
     if not os.path.exists(path):
         return None
     for line in open(path):
         cells = [c.strip() for c in line.strip().strip("|").split("|")]
-        if len(cells) >= 6 and cells[0] == kernel:
+        if len(cells) >= 7 and cells[0] == kernel and cells[1] == family:
             try:
-                rd, wr, alg = int(cells[2]), int(cells[3]), int(cells[4])
+                rd, wr, alg = int(cells[3]), int(cells[4]), int(cells[5])
             except ValueError:
                 continue
-            return {"bytes_per_launch": rd + wr, "dram_read": rd, "dram_write": wr, "algorithmic_bytes": alg, "layer": cells[1],
-                    "source": "profiles/dram_traffic.md (" + cells[5] + "): one ncu capture, not this run"}
+            return {"bytes_per_launch": rd + wr, "dram_read": rd, "dram_write": wr, "algorithmic_bytes": alg, "layer": cells[2],
+                    "source": "profiles/dram_traffic.md (" + cells[6] + "): one ncu capture of that layer, not this run"}
     return None
 
 
@@ -585,7 +585,7 @@ def main():
         kernel = {"exact_tensor_bound": "exact_tc_kernel", "exact_hbm_bound": "exact_tc_kernel", "top1": "top1_fused_kernel"}[dom]
         roof = {k: fams[dom][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
         roof.update({"kernel": kernel, "family": dom, "peak_source": peaks["source"], "families": fams,
-                     "traffic": traffic_from_profiles(kernel)})
+                     "traffic": traffic_from_profiles(kernel, dom)})
 
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
     e2e = None
