@@ -56,6 +56,9 @@
 #ifdef GACONV_TUNING
 #define GACONV_TL(slot, cond) do { if (tl && (cond)) tl[slot] = clock64(); if (P.timeline && threadIdx.x == 128) gaconv_tuning_stamps[(blockIdx.y * gridDim.x + blockIdx.x) & 1023][slot] = gaconv_globaltimer(); } while (0)
 __device__ unsigned long long gaconv_tuning_stamps[1024][8];
+// per launch (CTA (0,0)): {entry, dependency satisfied, exit, shape} in nanoseconds of the global timer
+__device__ unsigned long long gaconv_tuning_tc_log[4096][4];
+__device__ unsigned int gaconv_tuning_tc_log_n;
 __device__ __forceinline__ unsigned long long gaconv_globaltimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #else
 #define GACONV_TL(slot, cond) do { } while (0)
@@ -215,7 +218,18 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = s_tmem_base;
+#ifdef GACONV_TUNING
+    const unsigned long long t_in = gaconv_globaltimer();
+#endif
     pdl_wait_prior_grid();     // set-up done; from here on global memory of the previous kernel is read and written
+#ifdef GACONV_TUNING
+    __shared__ unsigned int s_log_i;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        s_log_i = atomicAdd(&gaconv_tuning_tc_log_n, 1u) & 4095u;
+        gaconv_tuning_tc_log[s_log_i][0] = t_in; gaconv_tuning_tc_log[s_log_i][1] = gaconv_globaltimer();
+        gaconv_tuning_tc_log[s_log_i][3] = ((unsigned long long)g.c << 40) | ((unsigned long long)g.k << 24) | ((unsigned long long)gridDim.x * gridDim.y << 8) | (unsigned)g.p;
+    }
+#endif
 #ifdef GACONV_TUNING
     long long* tl = (P.timeline && blockIdx.x == 0 && blockIdx.y == 0) ? reinterpret_cast<long long*>(status + 16) : nullptr;
 #endif
@@ -537,6 +551,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     if (cl > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     if (cl > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");      // peers may still be reading this CTA's block
     GACONV_TL(7, threadIdx.x == 0);
+#ifdef GACONV_TUNING
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) gaconv_tuning_tc_log[s_log_i][2] = gaconv_globaltimer();
+#endif
 }
 
 // dYt[n][j][k] = dY[n][k][j] for maps of fewer than 64 pixels (their rows are too short for the copy engine).
@@ -749,7 +766,7 @@ bool choose_splits(TcParams& P, const Geom& g, int tiles)
     if (cl == 0) return false;
     P.cl = cl;
     P.splits = splits;
-    P.reduce_parts = std::max(1, 2 * sm_count() / tiles);
+    P.reduce_parts = std::max(1, 2 * sms / tiles);          // the second kernel takes the same share of the GPU
     P.chunk_base = P.chunks / splits;
     P.chunk_rem = P.chunks - P.chunk_base * splits;
     return true;
@@ -1110,5 +1127,10 @@ cudaError_t launch_tc(const void* x, const void* dy, float* dw, float* partial, 
 extern "C" int gaconv_tuning_read_stamps(unsigned long long* host)
 {
     return (int)cudaMemcpyFromSymbol(host, gaconv_tuning_stamps, sizeof(gaconv_tuning_stamps));
+}
+extern "C" int gaconv_tuning_read_tc_log(unsigned long long* host, unsigned int* count)
+{
+    if (cudaMemcpyFromSymbol(count, gaconv_tuning_tc_log_n, sizeof(unsigned int)) != cudaSuccess) return 1;
+    return (int)cudaMemcpyFromSymbol(host, gaconv_tuning_tc_log, sizeof(gaconv_tuning_tc_log));
 }
 #endif

@@ -253,13 +253,32 @@ __device__ __forceinline__ void raw_to_float(const Raw4& r, const __nv_bfloat16*
 //   phase 3  after a cluster barrier, CTA j adds slice j of the block over the CL CTAs through
 //            distributed shared memory, in rank order, and writes alpha * total to dW.
 // No global scratch, no atomics; the order of every sum is fixed.
+#ifdef GACONV_TUNING
+// tuning builds: CTA (0,0) of every launch logs {entry, dependency satisfied, exit} in nanoseconds
+__device__ unsigned long long gaconv_tuning_top1_log[4096][4];
+__device__ unsigned int gaconv_tuning_top1_log_n;
+__device__ __forceinline__ unsigned long long tuning_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#endif
+
 template <typename T, bool VEC, bool WIDE>
 __global__ void __launch_bounds__(512, 2)
 top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x, int NJ)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+#ifdef GACONV_TUNING
+    const unsigned long long t_in = tuning_now();
+    const bool logger = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+    unsigned int log_i = 0;
+#endif
     pdl_wait_prior_grid();
+#ifdef GACONV_TUNING
+    if (logger) {
+        log_i = atomicAdd(&gaconv_tuning_top1_log_n, 1u) & 4095u;
+        gaconv_tuning_top1_log[log_i][0] = t_in; gaconv_tuning_top1_log[log_i][1] = tuning_now();
+        gaconv_tuning_top1_log[log_i][3] = ((unsigned long long)g.c << 32) | (unsigned)(g.k * 65536 + g.p);
+    }
+#endif
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int rsc = g.r * g.s * g.c;
     float* s_part = reinterpret_cast<float*>(smem_raw);                 // [rsc]
@@ -384,6 +403,9 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
         dw[k * g.ws_k + c * g.ws_c + r * g.ws_r + s * g.ws_s] = g.alpha * tot;
     }
     cluster.sync();     // peers may still be reading this CTA's block
+#ifdef GACONV_TUNING
+    if (logger) gaconv_tuning_top1_log[log_i][2] = tuning_now();
+#endif
 }
 
 // grid (chunks, K).  Each CTA owns the images [chunk*ipc, (chunk+1)*ipc) of one output channel and
@@ -552,7 +574,7 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     int nj = 1;
     // 512 threads (two CTAs per SM) where the grid still fits in one wave and the scan would otherwise need
     // two passes over the CTA's maps; measured: helps 32-channel layers, neutral or worse for 16 and 64
-    const int threads = (g.k >= 32 && (long long)cl * g.k <= 148 * 2) ? 512 : 256;
+    const int threads = (g.sm_budget == 0 && g.k >= 32 && (long long)cl * g.k <= 148 * 2) ? 512 : 256;
     const int groups = rsc / (WIDE ? 8 : vec_x ? 4 : 1);
     const int batch = (sizeof(T) == 4 || WIDE) ? 4 : 8;
     (void)batch;
@@ -574,6 +596,16 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     return e;
 }
 
+#ifdef GACONV_TUNING
+}  // namespace gaconv
+extern "C" int gaconv_tuning_read_top1_log(unsigned long long* host, unsigned int* count)
+{
+    if (cudaMemcpyFromSymbol(count, gaconv::gaconv_tuning_top1_log_n, sizeof(unsigned int)) != cudaSuccess) return 1;
+    return (int)cudaMemcpyFromSymbol(host, gaconv::gaconv_tuning_top1_log, sizeof(gaconv::gaconv_tuning_top1_log));
+}
+namespace gaconv {
+#endif
+
 cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream)
 {
     int cl = 1;
@@ -581,6 +613,10 @@ cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Ge
     // fewer, fatter CTAs when there are already plenty of channels: the whole grid should be resident
     // at once (four CTAs of 64 registers x 256 threads fit an SM)
     while (cl > 1 && (long long)cl * g.k > 148 * 4) cl /= 2;
+    // sharing the GPU with other layers (the caller gave an SM budget): about four CTAs per budgeted SM, so that the
+    // registers of several such kernels fit next to one another
+    if (g.sm_budget > 0)
+        while (cl > 1 && (long long)cl * g.k > 4LL * g.sm_budget) cl /= 2;
     const int ipc = (g.n + cl - 1) / cl;
     const MapScanShape m = map_scan_shape(g);
     if (g.bf16) {
