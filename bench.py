@@ -328,7 +328,7 @@ def main():
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtypes", default=None, help="comma list of bf16,f32 (default: the workload's)")
     ap.add_argument("--layer-iters", type=int, default=5, help="per-layer timing repetitions (median)")
-    ap.add_argument("--lanes", type=int, default=8, help="streams on which the layers of a step run next to one another (1..8)")
+    ap.add_argument("--lanes", type=int, default=12, help="streams on which the layers of a step run next to one another (1..16)")
     ap.add_argument("--budget-div", type=float, default=12.0, help="SM share of a layer in the step: 148 * roofline us / this")
     ap.add_argument("--budget-min", type=int, default=18)
     ap.add_argument("--budget-max", type=int, default=74)

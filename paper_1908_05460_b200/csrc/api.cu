@@ -431,7 +431,7 @@ gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t* s, int32_t la
 // ---- lanes: side streams on which the layers of a step run next to one another ----------------------
 namespace {
 
-constexpr int kMaxLanes = 8, kMaxLaneDevices = 64;
+constexpr int kMaxLanes = 16, kMaxLaneDevices = 64;
 struct LanePool {
     bool ready = false;
     cudaStream_t side[kMaxLanes - 1] = {};
