@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 METRIC = "dW-conv us/layer"
 UNIT = "us/layer"
 WORKLOADS = {0: "vgg19+resnet20+cnn2_cifar10_n128", 2: "resnet20_cifar10_n128", 3: "cnn2_cifar10_n128", 4: "vgg19_cifar10_n128"}
-ORACLE_SAMPLE_IMAGES = 32     # images per distinct layer shape that both oracle legs time (scaled to the batch): ~5 s of CPU work
+ORACLE_SAMPLE_IMAGES = 128    # images per distinct layer shape that both oracle legs time (the whole batch at N = 128): ~6 s of CPU work
 
 
 def workload_sets(config: int, batch: int, dtypes=None):

@@ -204,7 +204,7 @@ gaconv_status_t gaconv_schedule_run_layer(const gaconv_schedule_t *sched, int32_
  * per device), forked from `stream` when the call starts and joined back into it before it returns, so for the
  * caller the whole step is ordered like one operation on `stream` -- also inside a stream capture.  Layers of
  * different lanes overlap on the GPU, which hides the start-up and reduction latency of small layers; every
- * layer's result is bit for bit that of gaconv_schedule_run_layer.  lanes in 1..16; with lanes > 1 the
+ * layer's result is bit for bit that of gaconv_schedule_run_layer with the same descriptor.  lanes in 1..16; with lanes > 1 the
  * descriptors must carry distinct workspaces (GACONV_ERR_BAD_DESC otherwise).  x, dy, dw, descs: host arrays
  * of num_layers device pointers / descriptor pointers.  Calls on one device share the lanes: enqueueing from
  * several host threads is serialised. */
