@@ -606,6 +606,11 @@ def main():
         e2e = {"value": dist_util.us_per_layer(ms_e, passes, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": k2}
 
+    # bounded device waits that gave up leave a flag in the layer's workspace: none may be set after a clean run
+    timeouts = sum(1 for s in slots for d in (s.desc, s.step_desc) if B.gaconv_poll_async_status(d) != B.OK)
+    if timeouts:
+        print("warning: %d workspace status words report a device wait that gave up" % timeouts, file=sys.stderr)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -637,6 +642,7 @@ def main():
                    "l2": "inputs larger than L2: %.0f MB stream through between two uses of a buffer (method-major "
                          "order); per-layer timings stream over rotating input copies > 2.5x L2" % (input_bytes / 1e6)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "device_wait_timeouts": timeouts,
         "roofline": roof, "cpu_baseline": cpu,
         "breakdown_us": {"step_by_method": step_by_method, "streamed_sum_per_step": sum_us, "event_pair_overhead_us": empty_pair_us,
                          "exact_us_per_layer": sum_us["exact"] / passes, "top1_us_per_layer": sum_us["top1"] / passes,
