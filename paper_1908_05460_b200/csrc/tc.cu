@@ -150,6 +150,8 @@ struct TcParams {
     int rsplit;         // 1: a CTA handles ONE filter row (tile index carries r); N = s * 64
     int rc;             // filter rows per CTA: g.r, or 1 when rsplit
     int dual;           // 1 (only with rc == 1): two accumulators, issuer i takes the chunks with (index & 1) == i
+    int stack;          // 1: the R filter rows are stacked in M (row r of the filter = rows r*kb .. r*kb+kb-1 of the accumulator):
+                        //    A = R copies of the dY box, shifted by one image row each; B = the X rows of the chunk, no halo rows
     int issuers;        // MMA-issuing warps: min(R, 3), or 2 when dual; issuer i takes filter rows i, i+issuers, ...
     int slot_quads;     // float4 elements of one cluster slot (m rows x rc * s * ct columns)
     uint32_t qpr_magic; // ceil(2^32 / quads per row): quad index -> row by one multiply
@@ -159,6 +161,16 @@ struct TcParams {
 };
 
 constexpr int kMaxStages = 8;
+// accumulator row -> element offset of its output channel (and, when the filter rows are stacked in M, its filter
+// row) in dW; -1 for a row that holds nothing
+__device__ __forceinline__ int tc_row_offset(const TcParams& P, int k0, int row)
+{
+    const Geom& g = P.g;
+    if (!P.stack) return k0 + row < g.k ? (int)((k0 + row) * g.ws_k) : -1;
+    const int r = row / P.kb, kk = row - r * P.kb;
+    return (r < g.r && kk < g.k) ? (int)(kk * g.ws_k + r * g.ws_r) : -1;
+}
+
 constexpr int kMaxQuadCols = 7 * 256 / 4;      // rc <= 7 filter rows of at most 256 columns
 
 // R_T: filter rows (0 = take it from the geometry); KS_T: k-steps per A box (0 = from the plan).
@@ -177,6 +189,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     // its four channels exist (the last channel tile may be partial)
     __shared__ int s_coloff[kMaxQuadCols];
     __shared__ signed char s_colvalid[kMaxQuadCols];
+    __shared__ int s_rowoff[128];              // accumulator row -> offset in dW, or -1
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -196,6 +209,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     if (P.timeline && threadIdx.x == 128) gaconv_tuning_stamps[(blockIdx.y * gridDim.x + blockIdx.x) & 1023][1] = gaconv_globaltimer();
 #endif
     pdl_release_next_grid();
+    if (threadIdx.x < P.m) s_rowoff[threadIdx.x] = tc_row_offset(P, k0, threadIdx.x);
+    const int acc_rows = P.stack ? g.r * P.kb : min(P.m, g.k - k0);          // accumulator rows in use
     for (int cq = threadIdx.x; cq < (P.rc * nmma) >> 2; cq += blockDim.x) {
         const int col = cq << 2, rl = col / nmma, sc = col - rl * nmma, s_ = sc >> P.ct_shift, c = c0 + (sc & (P.ct - 1));
         s_coloff[cq] = (int)((r_lo + rl) * g.ws_r + s_ * g.ws_s + c * g.ws_c);
@@ -246,8 +261,8 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         if (whole_maps) { n0 = ch_begin * P.ci; p0 = 0; }
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
         const int planes = P.f32 && P.passes == 3 ? 2 : 1;
-        const uint32_t tx_bytes = planes * ((P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes);
-        const int n_a = P.f32 ? planes * P.a_subs : P.tiny ? P.m / 64 : P.by_image ? 1 : P.a_subs, n_all = n_a + planes * P.b_tiles;
+        const uint32_t tx_bytes = planes * ((P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.stack ? P.a_subs * g.r * P.kb * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes);
+        const int n_a = P.f32 ? planes * P.a_subs : P.tiny ? P.m / 64 : P.by_image ? 1 : P.stack ? g.r * P.a_subs : P.a_subs, n_all = n_a + planes * P.b_tiles;
         // what copy `lane` is: image and box of an A copy, or filter row and column shift of a B copy
         const int a_img = (P.tiny || P.by_image) ? 0 : lane / P.a_subs_img, a_sub = (P.tiny || P.by_image) ? 0 : lane - a_img * P.a_subs_img;
         const int b_idx = lane - n_a, b_rr = b_idx > 0 ? b_idx / g.s : 0, b_ss = b_idx > 0 ? b_idx - b_rr * g.s : 0;
@@ -280,6 +295,10 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                         tma_load_3d(sa + b * P.a_lbo, &map_dy, full, k0 + 64 * b, 0, n0);
                     } else if (P.by_image) {
                         tma_load_3d(sa, &map_dy, full, 0, k0, n0);               // ci whole maps in one box
+                    } else if (P.stack) {                                        // filter row rr: the box one image row earlier per row;
+                        const int rr = b / P.a_subs, sb_ = b - rr * P.a_subs;    // rows that leave the map read as zeros
+                        const int i = sb_ / P.a_subs_img, sub = sb_ - i * P.a_subs_img;
+                        tma_load_3d(sa + sb_ * P.a_sub_bytes + rr * P.kb * 128, &map_dy, full, (p0 - rr + g.pad_h) * g.q + 64 * sub, k0, n0 + i);
                     } else {                                                     // images past the batch read as zeros
                         const int i = b < 32 ? a_img : b / P.a_subs_img, sub = b < 32 ? a_sub : b - i * P.a_subs_img;
                         tma_load_3d(sa + b * P.a_sub_bytes, &map_dy, full, p0 * g.q + 64 * sub, k0, n0 + i);
@@ -289,7 +308,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                     if (P.tiny2) {                                               // dimensions (c, n, w, h)
                         tma_load_4d(sb, &map_x, full, c0, n0, -g.pad_w, r_lo - g.pad_h);
                     } else if (P.wide) {
-                        tma_load_4d(sb, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0);
+                        tma_load_4d(sb, &map_x, full, c0, -g.pad_w, P.stack ? p0 : p0 + r_lo - g.pad_h, n0);
                     } else if (P.halo) {
                         tma_load_4d(sb + j * P.b_tile_stride, &map_x, full, c0, j - g.pad_w, p0 - g.pad_h, n0);
                     } else {
@@ -401,7 +420,9 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     __syncwarp();
     const bool vec = g.ws_c == 1 && (g.c & 3) == 0;
     auto store_dw = [&](int row, int cq, const float4& t) {      // alpha * t -> the four elements of (row, quad column cq)
-        float* p = dw + (size_t)(k0 + row) * g.ws_k + s_coloff[cq];
+        const int ro = s_rowoff[row];
+        if (ro < 0) return;
+        float* p = dw + ro + s_coloff[cq];
         const int valid = s_colvalid[cq];
         const float a = g.alpha;
         if (vec && valid == 4) {
@@ -431,7 +452,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
                 // accumulator 0 (even chunks) + accumulator 1 (odd chunks).  M = 128: they sit side by side in the
                 // columns; M = 64: in the two 16-lane halves of each sub-partition (lane l and lane l + 16).
                 const bool has0 = nchunks > 0, has1 = nchunks > 1;
-                const bool row_ok = k0 + row < g.k && (P.m == 128 || lane < 16);
+                const bool row_ok = row < acc_rows && (P.m == 128 || lane < 16);
                 float* rrow = red + row * red_stride;
                 for (int pc = half; pc < pieces; pc += 4) {     // this warp: pieces pc and pc + 2
                     float v0[2][16], v1[2][16];
@@ -510,7 +531,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
     const int groups_per_tile = P.splits / cl, cgroup = split / cl;
     if (cl > 1) cluster.sync();
     GACONV_TL(5, threadIdx.x == 0);
-    const int rows = min(P.m, g.k - k0), cols = P.rc * nmma;
+    const int rows = acc_rows, cols = P.rc * nmma;
     const int q_per_row = cols >> 2, quads = rows * q_per_row;
     const int slice = (quads + cl - 1) / cl;
     const int f_begin = min(quads, rank * slice), f_end = min(quads, f_begin + slice);
@@ -606,7 +627,7 @@ reduce_slots_kernel(const float4* __restrict__ partial, float* __restrict__ dw, 
     __syncthreads();
     pdl_wait_prior_grid();
     const int groups = P.splits / P.cl;
-    const int quads = min(P.m, g.k - k0) * q_per_row;
+    const int quads = (P.stack ? g.r * P.kb : min(P.m, g.k - k0)) * q_per_row;
     const int part = (quads + (int)gridDim.x - 1) / (int)gridDim.x;
     const int p_begin = min(quads, (int)blockIdx.x * part), npart = min(quads, p_begin + part) - p_begin;
     int lg = 0;
@@ -633,7 +654,9 @@ reduce_slots_kernel(const float4* __restrict__ partial, float* __restrict__ dw, 
         }
         if (sl == 0 && q < npart) {
             const int f = p_begin + q, row = (int)__umulhi((uint32_t)f, P.qpr_magic), cq = f - row * q_per_row;
-            float* p = dw + (size_t)(k0 + row) * g.ws_k + s_coloff[cq];
+            const int ro = tc_row_offset(P, k0, row);
+            if (ro < 0) continue;
+            float* p = dw + ro + s_coloff[cq];
             const int valid = s_colvalid[cq];
             const float a = g.alpha;
             if (vec && valid == 4) {
@@ -801,13 +824,23 @@ bool plan_tc(const Geom& g, TcPlan* out)
     // cluster shrinks from 64 x R*S*64 floats (147 KB for 3x3) to a third, and that reduction, not the MMAs,
     // is what a small layer spends its time on.
     P.rsplit = (g.c >= 64 && g.r > 1 && env_int("GACONV_TC_RSPLIT", 1)) ? 1 : 0;
-    P.rc = P.rsplit ? 1 : g.r;
+    // Few output channels and narrow inputs (the 16- and 32-channel layers): the MMAs are tiny and the kernel is
+    // bound by how fast threads can issue them.  With "same" padding the R filter rows can share ONE MMA: row r
+    // of the filter becomes rows r*kb.. of M, fed by the dY box shifted by r image rows (the copy engine fills the
+    // rows that leave the map with zeros), against the same X rows.  R times fewer MMAs, and the single
+    // accumulator leaves room for the two-issuer scheme.
+    const int kb8 = (g.k + 7) / 8 * 8;
+    const bool stack = !P.rsplit && !small_map && g.r > 1 && g.r * kb8 <= 128 && g.stride_h == 1 && g.h == g.p &&
+                       (g.q % 16 == 0 || g.q == 8) && 64 % g.q == 0 && env_int("GACONV_TC_WIDE", 1) && env_int("GACONV_TC_STACK", 1);
+    P.stack = stack ? 1 : 0;
+    P.rc = (P.rsplit || stack) ? 1 : g.r;
     if (P.rsplit) P.m = g.k <= 64 ? 64 : 128;
+    if (stack) P.m = g.r * kb8 <= 64 ? 64 : 128;
     // One filter row per CTA means one accumulator and one issuing thread, which cannot keep the tensor pipe
     // busy (an MMA of N <= 256 executes in about the time one thread needs to issue it).  So the CTA keeps
     // two accumulators for the row and two issuers take alternate chunks.
     P.dual = (P.rc == 1 && env_int("GACONV_TC_DUAL", 1)) ? 1 : 0;
-    P.kb = (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
+    P.kb = stack ? kb8 : (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
     P.tiny = tiny ? 1 : 0;
     P.kpx = 16; P.passes = 1;
     P.by_image = small_map ? 1 : 0;
@@ -820,7 +853,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     if ((g.s * ct) % (P.m == 128 ? 16 : 8) != 0) return false;
     P.ct = ct;
     P.ct_shift = ct == 64 ? 6 : ct == 32 ? 5 : 4;
-    P.tiles_k = (g.k + P.m - 1) / P.m;
+    P.tiles_k = stack ? 1 : (g.k + P.m - 1) / P.m;
     P.tiles_c = (g.c + ct - 1) / ct;
     if (P.rsplit) halo = false;          // a single row needs no halo rows: its S tiles are loaded directly
     P.halo = halo ? 1 : 0;
@@ -840,7 +873,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     auto stage_bytes = [&](int ci, int bp, int* a_subs, int* tile_bytes, int* tile_stride) {
         const int px = ci * bp * g.q;
         *a_subs = tiny ? px / 64 : small_map ? ci : px / 64;
-        const int a_bytes = ((tiny ? (P.m / 64) * px * 128 : small_map ? P.kb * pq * 2 * ci : *a_subs * P.kb * 128) + 1023) / 1024 * 1024;
+        const int a_bytes = ((tiny ? (P.m / 64) * px * 128 : small_map ? P.kb * pq * 2 * ci : *a_subs * (stack ? P.m : P.kb) * 128) + 1023) / 1024 * 1024;
         const int rows = (halo || P.wide) ? bp + P.rc - 1 : bp;
         *tile_bytes = ci * rows * (P.wide ? g.q + g.s - 1 : g.q) * ct * 2;
         *tile_stride = (*tile_bytes + 1023) / 1024 * 1024;
@@ -879,7 +912,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.stage_bytes = (P.stage_bytes + 1023) / 1024 * 1024;
     P.a_subs = a_subs; P.b_tile_bytes = tb; P.b_tile_stride = ts;
     P.a_subs_img = (tiny || small_map) ? a_subs : a_subs / ci;
-    P.a_sub_bytes = tiny2 ? ci * g.q * 128 : tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : P.kb * 128;   // small maps: per image; one box carries ci of them
+    P.a_sub_bytes = tiny2 ? ci * g.q * 128 : tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : (stack ? P.m : P.kb) * 128;   // small maps: per image; one box carries ci of them
     P.b_lbo = tiny2 ? ci * 128 : P.wide ? ct * 2 : ts;
     P.b_sub_bytes = tiny2 ? (g.q + g.s - 1) * ci * 128 : P.wide ? (P.a_sub_px / g.q) * (g.q + g.s - 1) * ct * 2 : P.a_sub_px * ct * 2;
     P.a_k4_step = tiny ? (16 * 128) >> 4 : 2;
