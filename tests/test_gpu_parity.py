@@ -292,6 +292,12 @@ TC_SHAPES = [
     ConvLayer("tc 512->512@4 one CTA per tile, whole output", 8, 512, 4, 4, 512, 3, 3, 1, 1),
     ConvLayer("tc 512->512@2 one CTA per tile, whole output", 64, 512, 2, 2, 512, 3, 3, 1, 1),
     ConvLayer("tc 256->256@8 several images per chunk, ragged batch", 21, 256, 8, 8, 256, 3, 3, 1, 1),
+    # filter rows stacked in M (few output channels, "same" padding)
+    ConvLayer("tc stacked rows, k20 (rows of the last block unused)", 4, 24, 16, 16, 20, 3, 3, 1, 1),
+    ConvLayer("tc stacked rows, 5x5 k16", 3, 16, 16, 16, 16, 5, 5, 1, 2),
+    ConvLayer("tc stacked rows, 8x8 maps, several images per chunk, ragged batch", 21, 32, 8, 8, 24, 3, 3, 1, 1),
+    ConvLayer("tc stacked rows, k40 fills M = 128", 3, 16, 32, 32, 40, 3, 3, 1, 1),
+    ConvLayer("tc no padding: rows not stacked", 4, 16, 18, 18, 16, 3, 3, 1, 0),
 ]
 
 
