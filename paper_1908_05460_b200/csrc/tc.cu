@@ -869,11 +869,12 @@ bool plan_tc(const Geom& g, TcPlan* out)
 
     // chunk size: as many rows (or images) as fit the stage budget.  The hand-over of a stage costs the producer
     // and the issuer several hundred cycles each, so a stage should carry at least ~8 MMAs.
-    const int budget = env_int("GACONV_TC_STAGE_KB", 64) * 1024;
+    // (stacked rows: R copies of every dY box; 66 KB lets a 16-row chunk of the 16- and 32-channel layers fit, three stages)
+    const int budget = env_int("GACONV_TC_STAGE_KB", stack ? 66 : 64) * 1024;
     auto stage_bytes = [&](int ci, int bp, int* a_subs, int* tile_bytes, int* tile_stride) {
         const int px = ci * bp * g.q;
         *a_subs = tiny ? px / 64 : small_map ? ci : px / 64;
-        const int a_bytes = ((tiny ? (P.m / 64) * px * 128 : small_map ? P.kb * pq * 2 * ci : *a_subs * (stack ? P.m : P.kb) * 128) + 1023) / 1024 * 1024;
+        const int a_bytes = ((tiny ? (P.m / 64) * px * 128 : small_map ? P.kb * pq * 2 * ci : *a_subs * (stack ? g.r * P.kb : P.kb) * 128) + 1023) / 1024 * 1024;
         const int rows = (halo || P.wide) ? bp + P.rc - 1 : bp;
         *tile_bytes = ci * rows * (P.wide ? g.q + g.s - 1 : g.q) * ct * 2;
         *tile_stride = (*tile_bytes + 1023) / 1024 * 1024;
@@ -912,7 +913,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     P.stage_bytes = (P.stage_bytes + 1023) / 1024 * 1024;
     P.a_subs = a_subs; P.b_tile_bytes = tb; P.b_tile_stride = ts;
     P.a_subs_img = (tiny || small_map) ? a_subs : a_subs / ci;
-    P.a_sub_bytes = tiny2 ? ci * g.q * 128 : tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : (stack ? P.m : P.kb) * 128;   // small maps: per image; one box carries ci of them
+    P.a_sub_bytes = tiny2 ? ci * g.q * 128 : tiny ? 64 * 128 : small_map ? P.kb * pq * 2 : (stack ? g.r * P.kb : P.kb) * 128;   // small maps: per image; one box carries ci of them
     P.b_lbo = tiny2 ? ci * 128 : P.wide ? ct * 2 : ts;
     P.b_sub_bytes = tiny2 ? (g.q + g.s - 1) * ci * 128 : P.wide ? (P.a_sub_px / g.q) * (g.q + g.s - 1) * ct * 2 : P.a_sub_px * ct * 2;
     P.a_k4_step = tiny ? (16 * 128) >> 4 : 2;
