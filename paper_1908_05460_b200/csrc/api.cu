@@ -85,14 +85,17 @@ Top1Layout top1_layout(const Geom& g)
 
 struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; StemPlan sp; bool tc_ok, stem_ok; };
 // fp32 inputs take the tcgen05 kernel (TF32 MMAs on split operands) where the layer is wide enough for the
-// tensor cores to pay for the extra pass that splits the operands; the one-pass TF32 mode needs no split
-bool tc_f32_wanted(const Geom& g, int math, int algo) { return !g.bf16 && (math == GACONV_MATH_TF32 || algo == GACONV_ALGO_TENSOR || g.c >= 64); }
+// tensor cores to pay for the extra pass that splits the operands: 64 input channels, or 32 when the filter
+// rows share one MMA (measured: 32->32@16x16 18.7 us against 19.9 us on the warp-level path; without the
+// stacking 24 us); the one-pass TF32 mode needs no split
+bool tc_f32_wanted(const Geom& g, int math, int algo) { return !g.bf16 && (math == GACONV_MATH_TF32 || algo == GACONV_ALGO_TENSOR || g.c >= 32); }
 
 ExactLayout exact_layout(const Geom& g, int math, int algo)
 {
     ExactLayout L;
     L.dp = plan_direct(g);
     L.tc_ok = g.bf16 ? plan_tc(g, &L.tp) : (tc_f32_wanted(g, math, algo) && plan_tc_f32(g, math == GACONV_MATH_TF32 ? 1 : 3, &L.tp));
+    if (L.tc_ok && !g.bf16 && g.c < 64 && !L.tp.stacked_rows && math != GACONV_MATH_TF32 && algo != GACONV_ALGO_TENSOR) L.tc_ok = false;
     L.partial_off = kWsDataOffset;
     size_t partial = L.dp.partial_bytes;
     if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;

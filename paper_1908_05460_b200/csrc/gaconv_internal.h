@@ -129,6 +129,7 @@ struct TcPlan {
     size_t partial_bytes;
     size_t scratch_bytes;                   // extra device scratch (transposed dY for very small maps)
     bool reads_transposed_dy;               // the kernel's dY operand is the transposed copy dYt[n][pq][k] in the scratch
+    bool stacked_rows;                      // the filter rows share one MMA (stacked in M): few output channels, "same" padding
     alignas(8) unsigned char opaque[512];   // kernel parameters, private to tc.cu
 };
 bool plan_tc(const Geom& g, TcPlan* plan);   // false: shape not covered, use the direct kernel

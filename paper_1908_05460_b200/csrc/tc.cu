@@ -262,7 +262,7 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
         else { n0 = ch_begin / cpi; p0 = (ch_begin % cpi) * P.bp; }
         const int planes = P.f32 && P.passes == 3 ? 2 : 1;
         const uint32_t tx_bytes = planes * ((P.tiny ? (P.m / 64) * P.ci * g.p * g.q * 128 : P.stack ? P.a_subs * g.r * P.kb * 128 : P.a_subs * P.a_sub_bytes) + P.b_tiles * P.b_tile_bytes);
-        const int n_a = P.f32 ? planes * P.a_subs : P.tiny ? P.m / 64 : P.by_image ? 1 : P.stack ? g.r * P.a_subs : P.a_subs, n_all = n_a + planes * P.b_tiles;
+        const int n_a = P.f32 ? planes * (P.stack ? g.r : 1) * P.a_subs : P.tiny ? P.m / 64 : P.by_image ? 1 : P.stack ? g.r * P.a_subs : P.a_subs, n_all = n_a + planes * P.b_tiles;
         // what copy `lane` is: image and box of an A copy, or filter row and column shift of a B copy
         const int a_img = (P.tiny || P.by_image) ? 0 : lane / P.a_subs_img, a_sub = (P.tiny || P.by_image) ? 0 : lane - a_img * P.a_subs_img;
         const int b_idx = lane - n_a, b_rr = b_idx > 0 ? b_idx / g.s : 0, b_ss = b_idx > 0 ? b_idx - b_rr * g.s : 0;
@@ -282,11 +282,14 @@ exact_tc_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constan
             for (int b = lane; b < n_all; b += 32) {
                 if (P.f32) {                                                     // fp32: boxes of 32 pixels, one set per plane
                     if (b < n_a) {
-                        const int pl = b / P.a_subs, sub = b - pl * P.a_subs, i = sub / P.a_subs_img, sb_ = sub - i * P.a_subs_img;
-                        tma_load_4d(sa + pl * P.a_plane_bytes + sub * P.a_sub_bytes, &map_dy, full, p0 * g.q + P.a_sub_px * sb_, k0, n0 + i, pl);
+                        const int per_plane = (P.stack ? g.r : 1) * P.a_subs;   // (stacked: one box per filter row, one image row earlier each)
+                        const int pl = b / per_plane, rest = b - pl * per_plane, rr = rest / P.a_subs, sub = rest - rr * P.a_subs;
+                        const int i = sub / P.a_subs_img, sb_ = sub - i * P.a_subs_img;
+                        tma_load_4d(sa + pl * P.a_plane_bytes + sub * P.a_sub_bytes + rr * P.kb * 128, &map_dy, full,
+                                    (P.stack ? p0 - rr + g.pad_h : p0) * g.q + P.a_sub_px * sb_, k0, n0 + i, pl);
                     } else {
                         const int pl = b - n_a;
-                        tma_load_5d(sb + pl * P.b_plane_bytes, &map_x, full, c0, -g.pad_w, p0 + r_lo - g.pad_h, n0, pl);
+                        tma_load_5d(sb + pl * P.b_plane_bytes, &map_x, full, c0, -g.pad_w, P.stack ? p0 : p0 + r_lo - g.pad_h, n0, pl);
                     }
                 } else if (b < n_a) {
                     if (P.tiny2) {                                               // one box per 64-channel atom, [pixel][image][k]
@@ -949,6 +952,7 @@ bool plan_tc(const Geom& g, TcPlan* out)
     out->partial_bytes = splits / cl > 1 ? (size_t)tiles * (splits / cl) * P.slot_quads * 16 : 0;
     out->scratch_bytes = tiny ? (size_t)g.n * g.k * pq * 2 : 0;      // transposed copy of dY
     out->reads_transposed_dy = tiny;
+    out->stacked_rows = P.stack != 0;
     static_assert(sizeof(TcParams) <= sizeof(out->opaque), "TcPlan::opaque too small");
     memcpy(out->opaque, &P, sizeof(P));
     return encode_fn() != nullptr;
@@ -967,20 +971,26 @@ bool plan_tc_f32(const Geom& g, int passes, TcPlan* out)
     P.g = g;
     P.f32 = 1; P.passes = passes; P.kpx = 8;
     P.m = g.k <= 64 ? 64 : 128;
-    P.rsplit = g.r > 1 ? 1 : 0;
+    // few output channels and "same" padding: all filter rows stacked in M, as in the bf16 plan
+    const int kb8 = (g.k + 7) / 8 * 8;
+    const bool stack = g.r > 1 && g.r * kb8 <= 128 && g.h == g.p && env_int("GACONV_TC_STACK", 1);
+    P.stack = stack ? 1 : 0;
+    if (stack) P.m = g.r * kb8 <= 64 ? 64 : 128;
+    P.rsplit = (!stack && g.r > 1) ? 1 : 0;
     P.rc = 1; P.dual = 1; P.issuers = 2;
-    P.kb = g.k < P.m ? (g.k + 7) / 8 * 8 : P.m;
+    P.kb = stack ? kb8 : (g.k < P.m ? (g.k + 7) / 8 * 8 : P.m);
+    const int arows = stack ? g.r * kb8 : P.kb;          // rows of a dY sub-tile (32 pixels) in shared memory
     const int ct = 32;
     P.ct = ct; P.ct_shift = 5;
-    P.tiles_k = (g.k + P.m - 1) / P.m;
+    P.tiles_k = stack ? 1 : (g.k + P.m - 1) / P.m;
     P.tiles_c = (g.c + ct - 1) / ct;
     P.wide = 1; P.b_tiles = 1;
     P.a_sub_px = 32;
     P.a_swz = swz_code(128); P.b_swz = 1;               // B: 128-byte swizzle with 32-byte base (MN-major 32-bit elements)
     const int planes = passes == 3 ? 2 : 1;
-    const int budget = env_int("GACONV_TC_STAGE_KB", 64) * 1024, wt = g.q + g.s - 1;
+    const int budget = env_int("GACONV_TC_STAGE_KB", stack ? 66 : 64) * 1024, wt = g.q + g.s - 1;
     auto stage = [&](int ci, int bp, int* a_bytes, int* tile_bytes) {
-        *a_bytes = (ci * bp * g.q / 32 * P.kb * 128 + 1023) / 1024 * 1024;
+        *a_bytes = (ci * bp * g.q / 32 * arows * 128 + 1023) / 1024 * 1024;
         *tile_bytes = (ci * bp * wt * ct * 4 + 1023) / 1024 * 1024;
         return planes * (*a_bytes + *tile_bytes);
     };
@@ -993,7 +1003,7 @@ bool plan_tc_f32(const Geom& g, int passes, TcPlan* out)
     P.stage_bytes = stage(ci, bp, &ab, &tb);
     P.a_subs = ci * bp * g.q / 32;
     P.a_subs_img = P.a_subs / ci;
-    P.a_sub_bytes = P.kb * 128;
+    P.a_sub_bytes = arows * 128;
     P.a_k4_step = 2;                                    // eight fp32 pixels = 32 bytes
     P.a_lbo = 16;
     P.a_region_bytes = planes * ab;
@@ -1027,6 +1037,7 @@ bool plan_tc_f32(const Geom& g, int passes, TcPlan* out)
     // the two planes of each operand, [plane][elements]
     out->scratch_bytes = passes == 3 ? 2 * ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * pq) * 4 : 0;
     out->reads_transposed_dy = false;
+    out->stacked_rows = P.stack != 0;
     memcpy(out->opaque, &P, sizeof(P));
     return encode_fn() != nullptr;
 }
