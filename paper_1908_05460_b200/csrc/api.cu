@@ -95,7 +95,11 @@ ExactLayout exact_layout(const Geom& g, int math, int algo)
     ExactLayout L;
     L.dp = plan_direct(g);
     L.tc_ok = g.bf16 ? plan_tc(g, &L.tp) : (tc_f32_wanted(g, math, algo) && plan_tc_f32(g, math == GACONV_MATH_TF32 ? 1 : 3, &L.tp));
-    if (L.tc_ok && !g.bf16 && g.c < 64 && !L.tp.stacked_rows && math != GACONV_MATH_TF32 && algo != GACONV_ALGO_TENSOR) L.tc_ok = false;
+    // (32 channels: only with stacked rows and operands small enough that writing and re-reading their split planes
+    //  stays cheap -- 32->16@32x32 with 25 MB of inputs measured 36 us on this path)
+    const size_t in_bytes = ((size_t)g.n * g.c * g.h * g.w + (size_t)g.n * g.k * g.p * g.q) * 4;
+    if (L.tc_ok && !g.bf16 && g.c < 64 && (!L.tp.stacked_rows || in_bytes > ((size_t)12 << 20)) && math != GACONV_MATH_TF32 &&
+        algo != GACONV_ALGO_TENSOR) L.tc_ok = false;
     L.partial_off = kWsDataOffset;
     size_t partial = L.dp.partial_bytes;
     if (L.tc_ok && L.tp.partial_bytes > partial) partial = L.tp.partial_bytes;
