@@ -2,8 +2,11 @@
 // approximation-schedule driver (paper Section 2.5).  Every step of the path runs in this library's
 // kernels; there is no CPU or library fallback.
 #include <atomic>
+#include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
+#include <vector>
 
 #include "gaconv_internal.h"
 
@@ -55,6 +58,51 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     return GACONV_OK;
 }
 
+// ---- plans are kept: the planners run once per (problem, device), not once per call --------------------------------
+// A key is every field a plan depends on, plus the device (SM count and resident clusters differ between devices).
+struct PlanKey {
+    long long v[26];
+    bool operator==(const PlanKey& o) const { return memcmp(v, o.v, sizeof(v)) == 0; }
+};
+PlanKey plan_key(const Geom& g, int a, int b)
+{
+    int dev = 0;
+    cudaGetDevice(&dev);
+    uint32_t alpha_bits;
+    memcpy(&alpha_bits, &g.alpha, sizeof(alpha_bits));
+    return PlanKey{{g.n, g.c, g.h, g.w, g.k, g.r, g.s, g.p, g.q, g.stride_h, g.stride_w, g.pad_h, g.pad_w, g.xs_n, g.xs_c, g.xs_h,
+                    g.xs_w, g.ws_k, g.ws_c, g.ws_r, g.ws_s, g.bf16 ? 1 : 0, (long long)alpha_bits, g.sm_budget, ((long long)a << 32) | (uint32_t)b, dev}};
+}
+template <typename L>
+class PlanCache {
+public:
+    template <typename Build>
+    L get(const PlanKey& key, Build build)
+    {
+#ifndef GACONV_TUNING            // tuning builds read planner overrides from the environment on every call
+        {
+            std::lock_guard<std::mutex> lock(m_);
+            for (size_t i = 0; i < e_.size(); ++i)
+                if (e_[i].first == key) {
+                    if (i != 0) std::swap(e_[i], e_[i - 1]);       // frequently used entries drift to the front
+                    return e_[i != 0 ? i - 1 : 0].second;
+                }
+        }
+#endif
+        L made = build();
+#ifndef GACONV_TUNING
+        std::lock_guard<std::mutex> lock(m_);
+        if (e_.size() >= kMaxEntries) e_.pop_back();
+        e_.emplace_back(key, made);
+#endif
+        return made;
+    }
+private:
+    static constexpr size_t kMaxEntries = 256;
+    std::mutex m_;
+    std::vector<std::pair<PlanKey, L>> e_;
+};
+
 // Maps of at most 4x4 pixels with many channels: the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes,
 // the same number of bytes gathered from L2) cost more than the dense contraction on tensor cores, and with so few
 // pixels per map the sparse tensor is not that sparse (1 - 1/(PQ), Section 2.3).  Then the method is run
@@ -66,7 +114,7 @@ bool top1_dense_route(const Geom& g, TcPlan* tp)
 }
 
 struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, scratch_off, total; GatherPlan gp; TcPlan tp; bool dense; };
-Top1Layout top1_layout(const Geom& g)
+Top1Layout build_top1_layout(const Geom& g)
 {
     Top1Layout L;
     L.gp = plan_gather(g);
@@ -83,6 +131,12 @@ Top1Layout top1_layout(const Geom& g)
     return L;
 }
 
+Top1Layout top1_layout(const Geom& g)
+{
+    static PlanCache<Top1Layout> cache;
+    return cache.get(plan_key(g, 0, 0), [&] { return build_top1_layout(g); });
+}
+
 struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPlan tp; StemPlan sp; bool tc_ok, stem_ok; };
 // fp32 inputs take the tcgen05 kernel (TF32 MMAs on split operands) where the layer is wide enough for the
 // tensor cores to pay for the extra pass that splits the operands: 64 input channels, or 32 when the filter
@@ -90,7 +144,7 @@ struct ExactLayout { size_t partial_off, scratch_off, total; DirectPlan dp; TcPl
 // stacking 24 us); the one-pass TF32 mode needs no split
 bool tc_f32_wanted(const Geom& g, int math, int algo) { return !g.bf16 && (math == GACONV_MATH_TF32 || algo == GACONV_ALGO_TENSOR || g.c >= 32); }
 
-ExactLayout exact_layout(const Geom& g, int math, int algo)
+ExactLayout build_exact_layout(const Geom& g, int math, int algo)
 {
     ExactLayout L;
     L.dp = plan_direct(g);
@@ -108,6 +162,12 @@ ExactLayout exact_layout(const Geom& g, int math, int algo)
     L.scratch_off = align_up(L.partial_off + partial, 256);
     L.total = align_up(L.scratch_off + (L.tc_ok ? L.tp.scratch_bytes : 0), 256);
     return L;
+}
+
+ExactLayout exact_layout(const Geom& g, int math, int algo)
+{
+    static PlanCache<ExactLayout> cache;
+    return cache.get(plan_key(g, math, algo), [&] { return build_exact_layout(g, math, algo); });
 }
 
 // entries retained per map by the top-k method: desc->topk clamped to the map size; 0 = invalid
