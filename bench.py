@@ -449,6 +449,15 @@ def main():
         run_step = base_step
     for t in range(args.warmup):
         run_step(t)
+    # the inputs were generated on the host for seconds while the GPU sat idle: keep it busy for a quarter of a second
+    # more, so that the clocks are up when the timed region starts (extra untimed steps, beyond the W asked for)
+    extra_warm, t_spin = 0, time.perf_counter()
+    torch.cuda.synchronize()
+    while time.perf_counter() - t_spin < 0.25:
+        run_step(args.warmup + extra_warm)
+        extra_warm += 1
+        if extra_warm % 8 == 0:
+            torch.cuda.synchronize()
     barrier()
 
     # ---- timed region: exactly K steps ----
@@ -635,7 +644,7 @@ def main():
         "config": {"workload": "%s (%d layer passes x {exact, top1, zero, random}; sets: %s)"
                                % (WORKLOADS[args.config].replace("n128", "n%d" % args.batch), passes,
                                   ", ".join("%s %s" % ({2: "resnet20", 3: "cnn2", 4: "vgg19"}[c], "/".join(dn)) for c, _, dn in sets)),
-                   "layer_passes_per_step": passes, "cuda_graph": graph is not None, "lanes": args.lanes,
+                   "layer_passes_per_step": passes, "extra_warmup_steps": extra_warm, "cuda_graph": graph is not None, "lanes": args.lanes,
                    "parallelism": ("dp%d, one dW all-reduce per step" % world) if (args.allreduce and world > 1) else ("%d independent replicas" % world if world > 1 else "1 GPU"),
                    "sm_budget": "per layer min(%d, max(%d, 148 * roofline us / %g)) SMs in the step; whole GPU in the per-layer timings"
                                 % (args.budget_max, args.budget_min, args.budget_div),
