@@ -595,6 +595,15 @@ def main():
         roof = {k: fams[dom][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
         roof.update({"kernel": kernel, "family": dom, "peak_source": peaks["source"], "families": fams,
                      "traffic": traffic_from_profiles(kernel, dom)})
+        # the same ratio for the layers as they run in the step (sized for their SM share, overlapping on the lanes):
+        # sum of the layers' roofline times / the method's share of the replayed step
+        if step_by_method:
+            roof["in_step"] = {
+                "exact": {"sum_roof_us": sum(r["exact_roof_us"] for r in table), "step_us": step_by_method["exact"],
+                          "frac": sum(r["exact_roof_us"] for r in table) / step_by_method["exact"]},
+                "top1": {"sum_roof_us": sum(r["top1_bytes"] for r in table) / (peaks["hbm_gbs"] * 1e3), "step_us": step_by_method["top1"],
+                         "frac": sum(r["top1_bytes"] for r in table) / (peaks["hbm_gbs"] * 1e3) / step_by_method["top1"]},
+                "note": "layers overlap in the step, so these are throughput fractions of the whole GPU, not per-launch ones"}
 
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
     e2e = None
