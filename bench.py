@@ -401,7 +401,7 @@ def main():
                 s.budget = layer_sm_budget(l, s.eb, peaks, args)
                 s.step_desc = B.make_desc(l, s.dtype, alpha=1.0 / l.n, sm_budget=s.budget)
                 s.step_ws = B.attach_workspace(s.step_desc)
-                h2d += 2 * (s.x_host.numel() + s.dy_host.numel()) * s.eb      # exact and top-1 each copy their inputs
+                h2d += (s.x_host.numel() + s.dy_host.numel()) * s.eb          # a layer's inputs are copied once per step
                 d2h += 4 * s.dw.numel() * 4
                 slots.append(s)
     L = len(slots)
@@ -608,10 +608,27 @@ def main():
     # ---- end to end through the host-buffer entry point (H2D and D2H inside the timed region) ----
     e2e = None
     if not args.no_e2e:
+        # a layer's inputs cross the link once per step (with its exact gradient); the other three gradients of the layer
+        # reuse the device copies; every result is read back to the host
+        # Layers alternate between two streams (all calls of a layer on the same one), so that one layer's results go back
+        # to the host while the next layer's inputs come in; the host waits once, at the end of the step.  Each method's
+        # result has its own pinned host buffer.
+        e2e_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        for s in slots:
+            s.dw_hosts = [s.dw_host] + [torch.empty_like(s.dw_host).pin_memory() for _ in range(len(methods) - 1)]
+
         def e2e_step(t):
-            for _, m in methods:
-                for s in slots:
-                    B.gaconv_dw_from_host(m, s.x_host, s.dy_host, s.dw_host, s.x, s.dy, s.dw, s.desc, seed=t)
+            main = torch.cuda.current_stream()
+            for st in e2e_streams:
+                st.wait_stream(main)
+            for i, s in enumerate(slots):
+                for j, (_, m) in enumerate(methods):
+                    first = m == B.METHOD_EXACT
+                    B.gaconv_dw_from_host_async(m, s.x_host if first else None, s.dy_host if first else None, s.dw_hosts[j], s.x, s.dy,
+                                                s.dw, s.desc, seed=t, stream=e2e_streams[i & 1])
+            for st in e2e_streams:
+                main.wait_stream(st)
+            main.synchronize()          # the step's results are on the host
         e2e_step(0)
         barrier()
         k2 = max(1, min(args.steps, 3))

@@ -14,7 +14,8 @@
  *     are host memory (pinned for true asynchrony).  The library allocates no device memory and keeps
  *     no reference to any buffer after the call returns (the work itself is asynchronous, see below).
  *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it; no entry point
- *     synchronises the host except gaconv_poll_async_status and gaconv_dw_from_host's final wait.
+ *     synchronises the host except gaconv_poll_async_status and gaconv_dw_from_host's final wait
+ *     (gaconv_dw_from_host_async has none).
  *   - Validation errors are returned at once and enqueue nothing.
  *   - dw is overwritten (no accumulate-into).  It is always fp32.
  *   - Same inputs, descriptor and seed give bitwise identical outputs from run to run: every
@@ -168,8 +169,17 @@ gaconv_status_t gaconv_approx_select_topk(const void *dy, int32_t *idx, float *s
  * exact) with HOST inputs and output: copies x_host and dy_host into the caller's device staging
  * buffers x_dev and dy_dev, runs, copies dw_dev back into dw_host, and waits for the stream.  The
  * host-to-device and device-to-host transfers are part of the call.  The paper's operator has the
- * same shape: activations and gradients in, filter gradient out (Section 2.4). */
+ * same shape: activations and gradients in, filter gradient out (Section 2.4).  x_host and dy_host may
+ * both be NULL: x_dev and dy_dev are then used as they are (a step that takes several gradients of one
+ * layer -- say the exact one and an approximation -- copies the layer's inputs once). */
 gaconv_status_t gaconv_dw_from_host(int32_t method, const void *x_host, const void *dy_host, float *dw_host,
+                                    void *x_dev, void *dy_dev, float *dw_dev,
+                                    const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
+
+/* The same without the final wait: the three transfers and the kernels are enqueued on `stream` and the call
+ * returns; dw_host holds the result once the caller has synchronised with the stream.  Layers enqueued on different
+ * streams overlap their transfers in the two directions of the host link. */
+gaconv_status_t gaconv_dw_from_host_async(int32_t method, const void *x_host, const void *dy_host, float *dw_host,
                                     void *x_dev, void *dy_dev, float *dw_dev,
                                     const gaconv_conv_desc_t *desc, uint64_t seed, void *stream);
 

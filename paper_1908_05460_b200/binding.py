@@ -31,7 +31,7 @@ SCHED_EVERY_4TH_LAYER, SCHED_ALT_LAYER_ALT_BATCH, SCHED_ALL_LAYERS_EVERY_4TH_BAT
 
 EXPORTS = [
     "gaconv_status_string", "gaconv_launch_count", "gaconv_workspace_size", "gaconv_workspace_init", "gaconv_dw_exact",
-    "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_poll_async_status",
+    "gaconv_dw_approx", "gaconv_approx_select", "gaconv_dw_from_host", "gaconv_dw_from_host_async", "gaconv_poll_async_status",
     "gaconv_schedule_create", "gaconv_schedule_method", "gaconv_schedule_run_layer", "gaconv_schedule_run_step", "gaconv_schedule_destroy",
     "gaconv_dw_exact_static", "gaconv_static_scratch_bytes", "gaconv_poll_async_status_static", "gaconv_approx_select_topk",
 ]
@@ -78,6 +78,7 @@ def load():
     lib.gaconv_dw_approx.argtypes = [i32, vp, vp, vp, dp, u64, vp]
     lib.gaconv_approx_select.argtypes = [vp, vp, vp, vp, dp, vp]
     lib.gaconv_dw_from_host.argtypes = [i32, vp, vp, vp, vp, vp, vp, dp, u64, vp]
+    lib.gaconv_dw_from_host_async.argtypes = [i32, vp, vp, vp, vp, vp, vp, dp, u64, vp]
     lib.gaconv_poll_async_status.argtypes = [dp, vp]
     lib.gaconv_poll_async_status_static.argtypes = [vp]
     lib.gaconv_approx_select_topk.argtypes = [vp, vp, vp, dp, vp]
@@ -193,6 +194,12 @@ def gaconv_dw_from_host(method: int, x_host, dy_host, dw_host, x_dev, dy_dev, dw
                         stream=None):
     _check(load().gaconv_dw_from_host(method, _ptr(x_host), _ptr(dy_host), _ptr(dw_host), _ptr(x_dev), _ptr(dy_dev),
                                       _ptr(dw_dev), ctypes.byref(desc), seed, _stream(stream)), "gaconv_dw_from_host")
+
+
+def gaconv_dw_from_host_async(method: int, x_host, dy_host, dw_host, x_dev, dy_dev, dw_dev, desc: ConvDesc, seed: int = 0,
+                              stream=None):
+    _check(load().gaconv_dw_from_host_async(method, _ptr(x_host), _ptr(dy_host), _ptr(dw_host), _ptr(x_dev), _ptr(dy_dev),
+                                            _ptr(dw_dev), ctypes.byref(desc), seed, _stream(stream)), "gaconv_dw_from_host_async")
 
 
 def gaconv_poll_async_status(desc: ConvDesc, stream=None) -> int:

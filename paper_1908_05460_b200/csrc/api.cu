@@ -383,9 +383,9 @@ gaconv_status_t gaconv_approx_select_topk(const void* dy, int32_t* idx, float* s
     return launch_select_topk(dy, idx, sum, g, t, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
 }
 
-gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
+static gaconv_status_t dw_from_host(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
                                     void* x_dev, void* dy_dev, float* dw_dev, const gaconv_conv_desc_t* desc,
-                                    uint64_t seed, void* stream)
+                                    uint64_t seed, void* stream, bool wait)
 {
     Geom g;
     gaconv_status_t st = make_geom(desc, &g);
@@ -397,7 +397,8 @@ gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const vo
     if (method < GACONV_METHOD_EXACT || method > GACONV_METHOD_TOPK) return GACONV_ERR_BAD_DESC;
     if (!aligned16(dw_dev)) return GACONV_ERR_MISALIGNED;
     if (needs_inputs) {
-        if (x_host == nullptr || dy_host == nullptr || x_dev == nullptr || dy_dev == nullptr) return GACONV_ERR_NULL_POINTER;
+        // both host inputs NULL: the staging buffers already hold this layer's inputs (an earlier call of the step copied them)
+        if ((x_host == nullptr) != (dy_host == nullptr) || x_dev == nullptr || dy_dev == nullptr) return GACONV_ERR_NULL_POINTER;
         if (!aligned16(x_dev) || !aligned16(dy_dev)) return GACONV_ERR_MISALIGNED;
         if (method == GACONV_METHOD_EXACT && desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
         size_t need = 0;
@@ -411,8 +412,9 @@ gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const vo
             if (desc->algo == GACONV_ALGO_TENSOR && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
         }
         const size_t eb = g.bf16 ? 2 : 4;
-        if (cudaMemcpyAsync(x_dev, x_host, (size_t)g.n * g.c * g.h * g.w * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-            cudaMemcpyAsync(dy_dev, dy_host, (size_t)g.n * g.k * g.p * g.q * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+        if (x_host != nullptr &&
+            (cudaMemcpyAsync(x_dev, x_host, (size_t)g.n * g.c * g.h * g.w * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+             cudaMemcpyAsync(dy_dev, dy_host, (size_t)g.n * g.k * g.p * g.q * eb, cudaMemcpyHostToDevice, cs) != cudaSuccess))
             return GACONV_ERR_CUDA;
     }
     st = method == GACONV_METHOD_EXACT ? gaconv_dw_exact(x_dev, dy_dev, dw_dev, desc, stream)
@@ -420,7 +422,22 @@ gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const vo
     if (st != GACONV_OK) return st;
     if (cudaMemcpyAsync(dw_host, dw_dev, (size_t)g.k * g.c * g.r * g.s * sizeof(float), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
         return GACONV_ERR_CUDA;
+    if (!wait) return GACONV_OK;
     return cudaStreamSynchronize(cs) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+}
+
+gaconv_status_t gaconv_dw_from_host(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
+                                    void* x_dev, void* dy_dev, float* dw_dev, const gaconv_conv_desc_t* desc,
+                                    uint64_t seed, void* stream)
+{
+    return dw_from_host(method, x_host, dy_host, dw_host, x_dev, dy_dev, dw_dev, desc, seed, stream, true);
+}
+
+gaconv_status_t gaconv_dw_from_host_async(int32_t method, const void* x_host, const void* dy_host, float* dw_host,
+                                          void* x_dev, void* dy_dev, float* dw_dev, const gaconv_conv_desc_t* desc,
+                                          uint64_t seed, void* stream)
+{
+    return dw_from_host(method, x_host, dy_host, dw_host, x_dev, dy_dev, dw_dev, desc, seed, stream, false);
 }
 
 gaconv_status_t gaconv_poll_async_status(const gaconv_conv_desc_t* desc, void* stream)

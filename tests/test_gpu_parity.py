@@ -202,6 +202,18 @@ def test_from_host_entry_point():
     ref, dn = oracle.dw_top1(to_f64(x), to_f64(dy), oshape(layer))
     B.gaconv_dw_from_host(B.METHOD_TOP1, xh, dyh, out, g.x, g.dy, g.dw, g.desc)
     assert norm_err(I.krsc_to_kcrs(out).to(torch.float64).numpy(), ref, dn) <= TOL_F32
+    # no host inputs: the staging buffers are used as the previous call left them
+    out.fill_(float("nan"))
+    B.gaconv_dw_from_host(B.METHOD_TOP1, None, None, out, g.x, g.dy, g.dw, g.desc)
+    assert norm_err(I.krsc_to_kcrs(out).to(torch.float64).numpy(), ref, dn) <= TOL_F32
+    # the variant that does not wait: the result is on the host once the stream has been synchronised
+    out.fill_(float("nan"))
+    B.gaconv_dw_from_host_async(B.METHOD_TOP1, xh, dyh, out, g.x, g.dy, g.dw, g.desc)
+    torch.cuda.current_stream().synchronize()
+    assert norm_err(I.krsc_to_kcrs(out).to(torch.float64).numpy(), ref, dn) <= TOL_F32
+    with pytest.raises(B.GaconvError) as e:                               # one host input without the other
+        B.gaconv_dw_from_host(B.METHOD_TOP1, xh, None, out, g.x, g.dy, g.dw, g.desc)
+    assert e.value.status == B.ERR_NULL_POINTER
     assert B.gaconv_poll_async_status(g.desc) == B.OK
 
 
