@@ -329,6 +329,10 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
         int32_t* idx = reinterpret_cast<int32_t*>(ws + L.idx_off);
         float* sum = reinterpret_cast<float*>(ws + L.sum_off);
         if (launch_select_topk(dy, idx, sum, g, t, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        // the one-launch kernel of the top-1 method, fed with the selected list (t records per image), where its
+        // shared-memory block fits; else the ticketed gather kernel
+        if (top1_fused_supported(g) && (size_t)g.n * t * 16 <= 48 * 1024 && desc->algo != GACONV_ALGO_DIRECT)   // (16 bytes per record)
+            return launch_top1_fused(x, dy, dw, g, cs, idx, sum, t) == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
         if (launch_gather(x, idx, sum, dw, reinterpret_cast<float*>(ws + L.partial_off),
                           reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), g, L.gp, t, cs) != cudaSuccess)
             return GACONV_ERR_CUDA;

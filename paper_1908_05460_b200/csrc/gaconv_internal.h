@@ -89,7 +89,8 @@ cudaError_t launch_select_topk(const void* dy, int32_t* idx, float* sum, const G
 
 // ---- Algorithm 1 in one launch (selection + patch accumulate + cluster reduction) ----
 bool top1_fused_supported(const Geom& g);
-cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream);
+cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream,
+                              const int32_t* sel_idx = nullptr, const float* sel_sum = nullptr, int topk = 1);
 
 // ---- zero / random gradient ----
 cudaError_t launch_zero(float* dw, size_t count, cudaStream_t stream);

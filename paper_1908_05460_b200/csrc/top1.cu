@@ -262,7 +262,8 @@ __device__ __forceinline__ unsigned long long tuning_now() { unsigned long long 
 
 template <typename T, bool VEC, bool WIDE>
 __global__ void __launch_bounds__(512, 2)
-top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x, int NJ)
+top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ dw, Geom g, int ipc, int G, bool vec_x, int NJ,
+                  const int32_t* __restrict__ sel_idx, const float* __restrict__ sel_sum, int topk)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -285,15 +286,30 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
     // per image of this CTA, one 16-byte record: {element offset of the patch's top-left pixel (64 bits), the signed
     // sum (float bits), validity bits: bit r = patch row r lies inside the image, bit 16+s = patch column s does}
     uint4* s_rec = reinterpret_cast<uint4*>(smem_raw + (((size_t)rsc * 4 + 15) & ~(size_t)15));      // [ipc]
-    float* s_subs = reinterpret_cast<float*>(s_rec + ipc);              // [NJ][rsc] lane subtotals
+    float* s_subs = reinterpret_cast<float*>(s_rec + ipc * topk);       // [NJ][rsc] lane subtotals
 
     const int k = blockIdx.y, chunk = blockIdx.x, CL = gridDim.x;
     const int n0 = chunk * ipc;
     const int cnt = max(0, min(ipc, g.n - n0));
     const int pq = g.p * g.q;
 
-    // ---- phase 1: selection ----
-    {
+    // ---- phase 1: selection (or, for the top-k method, the list another kernel selected) ----
+    auto put_record = [&](int slot, int i, int j, float weight) {
+        const int h0 = (j / g.q) * g.stride_h - g.pad_h, w0 = (j % g.q) * g.stride_w - g.pad_w;
+        const long long base = (long long)i * g.xs_n + (long long)h0 * g.xs_h + (long long)w0 * g.xs_w;
+        uint32_t mask = 0;
+        for (int r = 0; r < g.r; ++r) mask |= (uint32_t)((unsigned)(h0 + r) < (unsigned)g.h) << r;
+        for (int c = 0; c < g.s; ++c) mask |= (uint32_t)((unsigned)(w0 + c) < (unsigned)g.w) << (16 + c);
+        s_rec[slot] = make_uint4((uint32_t)(unsigned long long)base, (uint32_t)((unsigned long long)base >> 32), __float_as_uint(weight), mask);
+    };
+    if (sel_idx != nullptr) {
+        // record (image i, entry t): the retained position with weight sum / topk; images in order, entries in order of selection
+        for (int e = threadIdx.x; e < cnt * topk; e += blockDim.x) {
+            const int i = e / topk;
+            const long long m = (long long)(n0 + i) * g.k + k;
+            put_record(e, i, sel_idx[m * topk + (e - i * topk)], sel_sum[m] / (float)topk);
+        }
+    } else {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         const int sub = lane & (G - 1), per_warp = 32 / G, per_pass = (blockDim.x >> 5) * per_warp;
         for (int base = 0; base < cnt; base += per_pass) {
@@ -301,16 +317,10 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
             const bool live = i < cnt;
             int best_j; float s;
             scan_map<T, VEC>(dy + ((long long)(n0 + (live ? i : 0)) * g.k + k) * pq, live, pq, G, sub, best_j, s);
-            if (live && sub == 0) {
-                const int h0 = (best_j / g.q) * g.stride_h - g.pad_h, w0 = (best_j % g.q) * g.stride_w - g.pad_w;
-                const long long base = (long long)i * g.xs_n + (long long)h0 * g.xs_h + (long long)w0 * g.xs_w;
-                uint32_t mask = 0;
-                for (int r = 0; r < g.r; ++r) mask |= (uint32_t)((unsigned)(h0 + r) < (unsigned)g.h) << r;
-                for (int c = 0; c < g.s; ++c) mask |= (uint32_t)((unsigned)(w0 + c) < (unsigned)g.w) << (16 + c);
-                s_rec[i] = make_uint4((uint32_t)(unsigned long long)base, (uint32_t)((unsigned long long)base >> 32), __float_as_uint(s), mask);
-            }
+            if (live && sub == 0) put_record(i, i, best_j, s);
         }
     }
+    const int nrec = cnt * topk;           // records of this CTA: one per image, or topk per image
     __syncthreads();
 
     // ---- phase 2: patch accumulate ----
@@ -334,7 +344,7 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
             float acc[NV];
 #pragma unroll
             for (int t = 0; t < NV; ++t) acc[t] = 0.f;
-            for (int i0 = j; i0 < cnt; i0 += BATCH * NJ) {
+            for (int i0 = j; i0 < nrec; i0 += BATCH * NJ) {
                 // BATCH loads are issued before any is consumed; they stay raw (two or four registers each)
                 // until then, so that the register allocator has no reason to serialise them.  A patch element
                 // outside the image contributes weight 0 times a zero that is not loaded.
@@ -343,7 +353,7 @@ top1_fused_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __re
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
                     const int i = i0 + u * NJ;
-                    const bool in = i < cnt;
+                    const bool in = i < nrec;
                     const uint4 rec = s_rec[in ? i : 0];
                     const bool ok = in && (rec.w & bits) == bits;
                     wsum[u] = ok ? __uint_as_float(rec.z) : 0.f;
@@ -566,7 +576,8 @@ bool top1_fused_supported(const Geom& g)
 }
 
 template <typename T, bool VEC, bool WIDE>
-static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom& g, int cl, int ipc, int G, cudaStream_t stream)
+static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom& g, int cl, int ipc, int G, cudaStream_t stream,
+                                  const int32_t* sel_idx = nullptr, const float* sel_sum = nullptr, int topk = 1)
 {
     // block of sums + per-image arrays + up to 16 lane subtotals when the block is small
     const int rsc = g.r * g.s * g.c;
@@ -578,9 +589,9 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     const int groups = rsc / (WIDE ? 8 : vec_x ? 4 : 1);
     const int batch = (sizeof(T) == 4 || WIDE) ? 4 : 8;
     (void)batch;
-    while (nj < 16 && nj * 2 <= ipc && nj * 2 * groups <= threads) nj *= 2;        // image lanes: as many as keep every item on its own thread
+    while (nj < 16 && nj * 2 <= ipc * topk && nj * 2 * groups <= threads) nj *= 2;        // image lanes: as many as keep every item on its own thread
     while (nj > 1 && (size_t)rsc * 4 * (1 + nj) > 150 * 1024) nj /= 2;              // the subtotals must fit shared memory
-    const size_t smem = (((size_t)rsc * 4 + 15) & ~(size_t)15) + (size_t)ipc * 16 + (nj > 1 ? (size_t)nj * rsc * 4 : 0) + 16;
+    const size_t smem = (((size_t)rsc * 4 + 15) & ~(size_t)15) + (size_t)ipc * topk * 16 + (nj > 1 ? (size_t)nj * rsc * 4 : 0) + 16;
     static size_t configured[64] = {};           // per device: the attribute belongs to the device's copy of the kernel
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -591,7 +602,8 @@ static cudaError_t launch_fused_t(const T* x, const T* dy, float* dw, const Geom
     }
     // lanes per map: few enough that one pass covers all the CTA's maps (their loads are then all in flight at once)
     while (G > 1 && G * ipc > threads) G /= 2;
-    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC, WIDE>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj);
+    cudaError_t e = launch_kernel(top1_fused_kernel<T, VEC, WIDE>, dim3(cl, g.k), dim3(threads), smem, stream, dim3(cl, 1, 1), x, dy, dw, g, ipc, G, vec_x, nj,
+                                  sel_idx, sel_sum, topk);
     note_launch();
     return e;
 }
@@ -606,7 +618,9 @@ extern "C" int gaconv_tuning_read_top1_log(unsigned long long* host, unsigned in
 namespace gaconv {
 #endif
 
-cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream)
+// sel_idx != nullptr: the top-k method -- selection was done by launch_select_topk; the kernel accumulates topk records per image
+cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Geom& g, cudaStream_t stream,
+                              const int32_t* sel_idx, const float* sel_sum, int topk)
 {
     int cl = 1;
     while (cl * 2 <= 8 && cl * 2 <= g.n) cl *= 2;
@@ -622,14 +636,14 @@ cudaError_t launch_top1_fused(const void* x, const void* dy, float* dw, const Ge
     if (g.bf16) {
         auto xx = static_cast<const __nv_bfloat16*>(x); auto dd = static_cast<const __nv_bfloat16*>(dy);
         const bool wide = g.xs_c == 1 && g.c % 8 == 0 && g.xs_w % 8 == 0;     // 16-byte aligned groups of eight channels
-        if (wide) return m.vec ? launch_fused_t<__nv_bfloat16, true, true>(xx, dd, dw, g, cl, ipc, m.G, stream)
-                               : launch_fused_t<__nv_bfloat16, false, true>(xx, dd, dw, g, cl, ipc, m.G, stream);
-        return m.vec ? launch_fused_t<__nv_bfloat16, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream)
-                     : launch_fused_t<__nv_bfloat16, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
+        if (wide) return m.vec ? launch_fused_t<__nv_bfloat16, true, true>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk)
+                               : launch_fused_t<__nv_bfloat16, false, true>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk);
+        return m.vec ? launch_fused_t<__nv_bfloat16, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk)
+                     : launch_fused_t<__nv_bfloat16, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk);
     }
     auto xx = static_cast<const float*>(x); auto dd = static_cast<const float*>(dy);
-    return m.vec ? launch_fused_t<float, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream)
-                 : launch_fused_t<float, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream);
+    return m.vec ? launch_fused_t<float, true, false>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk)
+                 : launch_fused_t<float, false, false>(xx, dd, dw, g, cl, ipc, m.G, stream, sel_idx, sel_sum, topk);
 }
 
 }  // namespace gaconv

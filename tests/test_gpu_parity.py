@@ -540,6 +540,9 @@ def test_topk_matches_oracle(li, topk):
         got = g.approx(B.METHOD_TOPK)
         assert norm_err(got, ref, dn) <= TOL_F32
         np.testing.assert_array_equal(got, g.approx(B.METHOD_TOPK))             # reproducible
+        # the ticketed gather kernel (what shapes beyond the one-launch kernel's shared memory take)
+        gd = GpuLayer(layer, dtype, x, dy, alpha=0.5, topk=topk, algo=B.ALGO_DIRECT)
+        assert norm_err(gd.approx(B.METHOD_TOPK), ref, dn) <= TOL_F32
         if topk == 1:
             ref1, dn1 = oracle.dw_top1(xd, dyd, oshape(layer), 0.5)
             assert norm_err(got, ref1, dn1) <= TOL_F32
