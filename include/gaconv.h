@@ -43,7 +43,8 @@ typedef enum {
 } gaconv_status_t;
 
 typedef enum { GACONV_F32 = 0, GACONV_BF16 = 1 } gaconv_dtype_t;            /* of x and dy            */
-typedef enum { GACONV_X_NHWC = 0, GACONV_X_NCHW = 1 } gaconv_x_layout_t;    /* NHWC: Section 2.4     */
+typedef enum { GACONV_X_NHWC = 0, GACONV_X_NCHW = 1 } gaconv_x_layout_t;    /* NHWC: Section 2.4; NCHW is transposed once
+                                                                               into the workspace where a fast kernel applies */
 typedef enum { GACONV_DY_NKPQ = 0 } gaconv_dy_layout_t;                     /* = N C_o H W           */
 /* KRSC = C_o K K C_i (the layout of the paper's kernel, Section 2.4), KCRS = the frameworks' filter
  * layout, RSCK = K K C_i C_o (the order in which Section 2.4 first writes df) */

@@ -207,6 +207,60 @@ uint64_t splitmix64(uint64_t x)
     return z ^ (z >> 31);
 }
 
+// ---- N x C x H x W activations --------------------------------------------------------------------------------
+// The fast kernels (tensor-core, stem, vectorised gather) read channels-last activations.  Where one of them serves
+// the channels-last version of the problem, an N x C x H x W input is transposed once into the tail of the workspace
+// and the call continues as a channels-last call; otherwise (odd shapes, GACONV_ALGO_DIRECT) the FP32-pipe and
+// scalar-gather kernels read it in place.  Returns the inner (channels-last) workspace size, or 0 for "in place".
+size_t nchw_relayout_inner_bytes(const gaconv_conv_desc_t* desc, int32_t method)
+{
+    if (desc->x_layout != GACONV_X_NCHW || desc->c < 2 || desc->algo == GACONV_ALGO_DIRECT) return 0;
+    gaconv_conv_desc_t inner = *desc;
+    inner.x_layout = GACONV_X_NHWC;
+    Geom gi;
+    if (make_geom(&inner, &gi) != GACONV_OK) return 0;
+    if (method == GACONV_METHOD_EXACT) {
+        const ExactLayout L = exact_layout(gi, desc->math, desc->algo);
+        if (!(L.tc_ok || L.stem_ok || direct_mma_supported(gi, L.dp))) return 0;
+        return L.total;
+    }
+    if (method == GACONV_METHOD_TOP1) {
+        const Top1Layout L = top1_layout(gi);
+        if (!(L.dense || (top1_fused_supported(gi) && gi.c % 4 == 0))) return 0;
+        return L.total;
+    }
+    if (method == GACONV_METHOD_TOPK) {
+        const int t = topk_of(desc, gi);
+        if (t < 1 || !(top1_fused_supported(gi) && gi.c % 4 == 0)) return 0;
+        return topk_layout(gi, t).total;
+    }
+    return 0;
+}
+size_t x_bytes_of(const gaconv_conv_desc_t* d) { return (size_t)d->n * d->c * d->h * d->w * (d->in_dtype == GACONV_BF16 ? 2 : 4); }
+
+// Transposes x into the workspace tail and fills `inner` (a channels-last copy of the descriptor whose workspace is
+// the head).  GACONV_OK with *x_out == nullptr means "no relayout: go on in place".
+gaconv_status_t nchw_relayout(const void* x, const gaconv_conv_desc_t* desc, int32_t method, cudaStream_t cs,
+                              gaconv_conv_desc_t* inner, const void** x_out)
+{
+    *x_out = nullptr;
+    const size_t inner_bytes = nchw_relayout_inner_bytes(desc, method);
+    if (inner_bytes == 0) return GACONV_OK;
+    const size_t head = align_up(inner_bytes, 256);
+    gaconv_status_t st = check_ws(desc, head + x_bytes_of(desc));
+    if (st != GACONV_OK) return st;
+    Geom g;
+    st = make_geom(desc, &g);
+    if (st != GACONV_OK) return st;
+    void* xt = static_cast<char*>(desc->workspace) + head;
+    if (launch_nchw_to_nhwc(x, xt, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+    *inner = *desc;
+    inner->x_layout = GACONV_X_NHWC;
+    inner->workspace_bytes = head;
+    *x_out = xt;
+    return GACONV_OK;
+}
+
 }  // namespace
 
 struct gaconv_schedule {
@@ -241,6 +295,10 @@ gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t me
     Geom g;
     gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
+    if (const size_t inner = nchw_relayout_inner_bytes(desc, method)) {      // the channels-last call's scratch, then the transposed X
+        *bytes = align_up(inner, 256) + x_bytes_of(desc);
+        return GACONV_OK;
+    }
     switch (method) {
         case GACONV_METHOD_EXACT: *bytes = exact_layout(g, desc->math, desc->algo).total; return GACONV_OK;
         case GACONV_METHOD_TOP1: *bytes = top1_layout(g).total; return GACONV_OK;
@@ -273,6 +331,13 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
+    {
+        gaconv_conv_desc_t inner;
+        const void* xt = nullptr;
+        st = nchw_relayout(x, desc, GACONV_METHOD_EXACT, static_cast<cudaStream_t>(stream), &inner, &xt);
+        if (st != GACONV_OK) return st;
+        if (xt != nullptr) return gaconv_dw_exact(xt, dy, dw, &inner, stream);
+    }
     const ExactLayout L = exact_layout(g, desc->math, desc->algo);
     const bool mma_ok = direct_mma_supported(g, L.dp);
     if (desc->math == GACONV_MATH_TF32 && !mma_ok && !L.tc_ok) return GACONV_ERR_UNSUPPORTED;
@@ -318,6 +383,13 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     if (method != GACONV_METHOD_TOP1 && method != GACONV_METHOD_TOPK) return GACONV_ERR_BAD_DESC;
     if (x == nullptr || dy == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy)) return GACONV_ERR_MISALIGNED;
+    {
+        gaconv_conv_desc_t inner;
+        const void* xt = nullptr;
+        st = nchw_relayout(x, desc, method, cs, &inner, &xt);
+        if (st != GACONV_OK) return st;
+        if (xt != nullptr) return gaconv_dw_approx(method, xt, dy, dw, &inner, seed, stream);
+    }
     if (method == GACONV_METHOD_TOPK) {
         // selection of the topk largest magnitudes per map, then the patch accumulation over the retained entries
         const int t = topk_of(desc, g);

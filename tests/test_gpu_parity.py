@@ -107,6 +107,41 @@ def test_other_layouts(x_layout, dw_layout):
     assert np.max(np.abs(g.approx(B.METHOD_RANDOM, seed=5) * (0.25 * 128) - z)) < 1e-5 * 0.25 * 8
 
 
+# ---- N x C x H x W activations on shapes the fast kernels serve: one transposing pass, then the channels-last route ----
+NCHW_SHAPES = [
+    ConvLayer("nchw 16->16@32", 6, 16, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("nchw 64->64@8", 9, 64, 8, 8, 64, 3, 3, 1, 1),
+    ConvLayer("nchw 3->16@32 stem", 5, 3, 32, 32, 16, 3, 3, 1, 1),
+    ConvLayer("nchw 40->24@16 ragged channels", 4, 40, 16, 16, 24, 3, 3, 1, 1),
+    ConvLayer("nchw 256->64@4 small maps", 5, 256, 4, 4, 64, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("li", range(len(NCHW_SHAPES)), ids=[l.name for l in NCHW_SHAPES])
+def test_nchw_activations_take_the_fast_kernels_through_one_transposing_pass(li, dtype):
+    layer = NCHW_SHAPES[li]
+    x, dy = _inputs(layer, dtype, 45 + li)
+    xd, dyd = to_f64(x), to_f64(dy)
+    g = GpuLayer(layer, dtype, x, dy, x_layout=B.X_NCHW, alpha=0.5, topk=3)
+    nhwc = GpuLayer(layer, dtype, x, dy, alpha=0.5, topk=3)
+    ref, dn = oracle.dw_exact(xd, dyd, oshape(layer), 0.5)
+    got = g.exact()
+    assert norm_err(got, ref, dn) <= tol(dtype)
+    np.testing.assert_array_equal(got, nhwc.exact())                 # the same kernels on the same values
+    ref, dn = oracle.dw_top1(xd, dyd, oshape(layer), 0.5)
+    got = g.approx(B.METHOD_TOP1)
+    assert norm_err(got, ref, dn) <= top1_bound(layer, dtype)
+    np.testing.assert_array_equal(got, nhwc.approx(B.METHOD_TOP1))
+    ref, dn = oracle.dw_topk(xd, dyd, oshape(layer), 3, 0.5)
+    assert norm_err(g.approx(B.METHOD_TOPK), ref, dn) <= TOL_F32
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+    # read in place when asked for the FP32-pipe kernel
+    inplace = GpuLayer(layer, dtype, x, dy, x_layout=B.X_NCHW, alpha=0.5, algo=B.ALGO_DIRECT)
+    ref, dn = oracle.dw_exact(xd, dyd, oshape(layer), 0.5)
+    assert norm_err(inplace.exact(), ref, dn) <= tol(dtype)
+
+
 def test_selection_ties_and_planted_maxima():
     layer = ConvLayer("ties", 4, 2, 32, 32, 8, 3, 3, 1, 1)
     for dtype in DTYPES:
