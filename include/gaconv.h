@@ -45,7 +45,9 @@ typedef enum {
 typedef enum { GACONV_F32 = 0, GACONV_BF16 = 1 } gaconv_dtype_t;            /* of x and dy            */
 typedef enum { GACONV_X_NHWC = 0, GACONV_X_NCHW = 1 } gaconv_x_layout_t;    /* NHWC: Section 2.4; NCHW is transposed once
                                                                                into the workspace where a fast kernel applies */
-typedef enum { GACONV_DY_NKPQ = 0 } gaconv_dy_layout_t;                     /* = N C_o H W           */
+typedef enum { GACONV_DY_NKPQ = 0, GACONV_DY_NPQK = 1 } gaconv_dy_layout_t;  /* NKPQ = N C_o H W (Section 2.4); NPQK (channels
+                                                                               last) is transposed once into the workspace.
+                                                                               The selection-only entry points take NKPQ only */
 /* KRSC = C_o K K C_i (the layout of the paper's kernel, Section 2.4), KCRS = the frameworks' filter
  * layout, RSCK = K K C_i C_o (the order in which Section 2.4 first writes df) */
 typedef enum { GACONV_DW_KRSC = 0, GACONV_DW_KCRS = 1, GACONV_DW_RSCK = 2 } gaconv_dw_layout_t;

@@ -20,7 +20,7 @@ OK = 0
 ERR_NULL_POINTER, ERR_BAD_DESC, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = range(1, 8)
 F32, BF16 = 0, 1
 X_NHWC, X_NCHW = 0, 1
-DY_NKPQ = 0
+DY_NKPQ, DY_NPQK = 0, 1
 DW_KRSC, DW_KCRS, DW_RSCK = 0, 1, 2
 METHOD_EXACT, METHOD_ZERO, METHOD_RANDOM, METHOD_TOP1, METHOD_TOPK = -1, 0, 1, 2, 3
 MAX_TOPK = 16
@@ -124,14 +124,14 @@ def _stream(stream):
 
 
 def make_desc(layer: ConvLayer, dtype: torch.dtype, *, x_layout=X_NHWC, dw_layout=DW_KRSC, alpha=1.0,
-              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO, topk=1, sm_budget=0) -> ConvDesc:
+              rand_std=1.0 / 128, math=MATH_DEFAULT, algo=ALGO_AUTO, topk=1, sm_budget=0, dy_layout=DY_NKPQ) -> ConvDesc:
     d = ConvDesc()
     d.struct_size = ctypes.sizeof(ConvDesc)
     d.n, d.c, d.h, d.w, d.k, d.r, d.s = layer.n, layer.c, layer.h, layer.w, layer.k, layer.r, layer.s
     d.stride_h = d.stride_w = layer.stride
     d.pad_h = d.pad_w = layer.pad
     d.in_dtype = BF16 if dtype == torch.bfloat16 else F32
-    d.x_layout, d.dy_layout, d.dw_layout = x_layout, DY_NKPQ, dw_layout
+    d.x_layout, d.dy_layout, d.dw_layout = x_layout, dy_layout, dw_layout
     d.math, d.algo, d.topk, d.sm_budget = math, algo, topk, sm_budget
     d.alpha, d.rand_std = alpha, rand_std
     d.workspace, d.workspace_bytes = None, 0

@@ -28,7 +28,7 @@ gaconv_status_t make_geom(const gaconv_conv_desc_t* d, Geom* g)
     if (d->h + 2 * d->pad_h < d->r || d->w + 2 * d->pad_w < d->s) return GACONV_ERR_BAD_DESC;
     if (d->in_dtype != GACONV_F32 && d->in_dtype != GACONV_BF16) return GACONV_ERR_BAD_DESC;
     if (d->x_layout != GACONV_X_NHWC && d->x_layout != GACONV_X_NCHW) return GACONV_ERR_BAD_DESC;
-    if (d->dy_layout != GACONV_DY_NKPQ) return GACONV_ERR_BAD_DESC;
+    if (d->dy_layout != GACONV_DY_NKPQ && d->dy_layout != GACONV_DY_NPQK) return GACONV_ERR_BAD_DESC;
     if (d->dw_layout != GACONV_DW_KRSC && d->dw_layout != GACONV_DW_KCRS && d->dw_layout != GACONV_DW_RSCK) return GACONV_ERR_BAD_DESC;
     if (d->math != GACONV_MATH_DEFAULT && d->math != GACONV_MATH_TF32) return GACONV_ERR_BAD_DESC;
     if (d->algo < GACONV_ALGO_AUTO || d->algo > GACONV_ALGO_TENSOR) return GACONV_ERR_BAD_DESC;
@@ -207,57 +207,97 @@ uint64_t splitmix64(uint64_t x)
     return z ^ (z >> 31);
 }
 
-// ---- N x C x H x W activations --------------------------------------------------------------------------------
-// The fast kernels (tensor-core, stem, vectorised gather) read channels-last activations.  Where one of them serves
-// the channels-last version of the problem, an N x C x H x W input is transposed once into the tail of the workspace
-// and the call continues as a channels-last call; otherwise (odd shapes, GACONV_ALGO_DIRECT) the FP32-pipe and
-// scalar-gather kernels read it in place.  Returns the inner (channels-last) workspace size, or 0 for "in place".
-size_t nchw_relayout_inner_bytes(const gaconv_conv_desc_t* desc, int32_t method)
+// ---- operand layouts other than the kernels' own ---------------------------------------------------------------
+// The fast kernels (tensor-core, stem, vectorised gather) read channels-last activations, and every kernel reads dY
+// as N x K x P x Q.  An N x P x Q x K gradient (what a channels-last framework hands over) is always transposed into
+// the tail of the workspace; an N x C x H x W input is transposed where a fast kernel serves the channels-last
+// version of the problem, and read in place by the FP32-pipe and scalar-gather kernels otherwise (odd shapes,
+// GACONV_ALGO_DIRECT).  The call then continues with an inner descriptor in the kernels' layouts whose workspace is
+// the head of the caller's.
+struct Relayout { size_t inner_bytes; bool move_x, move_dy; gaconv_conv_desc_t inner; };
+size_t x_bytes_of(const gaconv_conv_desc_t* d) { return (size_t)d->n * d->c * d->h * d->w * (d->in_dtype == GACONV_BF16 ? 2 : 4); }
+size_t dy_bytes_of(const Geom& g) { return (size_t)g.n * g.k * g.p * g.q * (g.bf16 ? 2 : 4); }
+
+// workspace of a call in the kernels' own dY layout (x in either layout); 0 with *ok = false when the descriptor is bad
+size_t native_ws_bytes(const gaconv_conv_desc_t* desc, const Geom& g, int32_t method, bool* ok)
 {
-    if (desc->x_layout != GACONV_X_NCHW || desc->c < 2 || desc->algo == GACONV_ALGO_DIRECT) return 0;
-    gaconv_conv_desc_t inner = *desc;
-    inner.x_layout = GACONV_X_NHWC;
-    Geom gi;
-    if (make_geom(&inner, &gi) != GACONV_OK) return 0;
-    if (method == GACONV_METHOD_EXACT) {
-        const ExactLayout L = exact_layout(gi, desc->math, desc->algo);
-        if (!(L.tc_ok || L.stem_ok || direct_mma_supported(gi, L.dp))) return 0;
-        return L.total;
+    *ok = true;
+    switch (method) {
+        case GACONV_METHOD_EXACT: return exact_layout(g, desc->math, desc->algo).total;
+        case GACONV_METHOD_TOP1: return top1_layout(g).total;
+        case GACONV_METHOD_TOPK: {
+            const int t = topk_of(desc, g);
+            if (t < 1) { *ok = false; return 0; }
+            return topk_layout(g, t).total;
+        }
+        case GACONV_METHOD_ZERO:
+        case GACONV_METHOD_RANDOM: return kWsDataOffset;
     }
-    if (method == GACONV_METHOD_TOP1) {
-        const Top1Layout L = top1_layout(gi);
-        if (!(L.dense || (top1_fused_supported(gi) && gi.c % 4 == 0))) return 0;
-        return L.total;
-    }
-    if (method == GACONV_METHOD_TOPK) {
-        const int t = topk_of(desc, gi);
-        if (t < 1 || !(top1_fused_supported(gi) && gi.c % 4 == 0)) return 0;
-        return topk_layout(gi, t).total;
-    }
+    *ok = false;
     return 0;
 }
-size_t x_bytes_of(const gaconv_conv_desc_t* d) { return (size_t)d->n * d->c * d->h * d->w * (d->in_dtype == GACONV_BF16 ? 2 : 4); }
 
-// Transposes x into the workspace tail and fills `inner` (a channels-last copy of the descriptor whose workspace is
-// the head).  GACONV_OK with *x_out == nullptr means "no relayout: go on in place".
-gaconv_status_t nchw_relayout(const void* x, const gaconv_conv_desc_t* desc, int32_t method, cudaStream_t cs,
-                              gaconv_conv_desc_t* inner, const void** x_out)
+// which operands move, and the inner call's workspace size; move_x == move_dy == false: the call runs as it is
+Relayout plan_relayout(const gaconv_conv_desc_t* desc, int32_t method)
 {
-    *x_out = nullptr;
-    const size_t inner_bytes = nchw_relayout_inner_bytes(desc, method);
-    if (inner_bytes == 0) return GACONV_OK;
-    const size_t head = align_up(inner_bytes, 256);
-    gaconv_status_t st = check_ws(desc, head + x_bytes_of(desc));
-    if (st != GACONV_OK) return st;
+    Relayout R{};
+    R.inner = *desc;
+    const bool reads_inputs = method == GACONV_METHOD_EXACT || method == GACONV_METHOD_TOP1 || method == GACONV_METHOD_TOPK;
+    if (!reads_inputs) return R;
+    R.move_dy = desc->dy_layout == GACONV_DY_NPQK && desc->k > 1 && (long long)desc->h * desc->w > 0;
+    R.inner.dy_layout = GACONV_DY_NKPQ;
+    if (desc->x_layout == GACONV_X_NCHW && desc->c >= 2 && desc->algo != GACONV_ALGO_DIRECT) {
+        gaconv_conv_desc_t cl = R.inner;
+        cl.x_layout = GACONV_X_NHWC;
+        Geom gi;
+        if (make_geom(&cl, &gi) == GACONV_OK) {
+            if (method == GACONV_METHOD_EXACT) {
+                const ExactLayout L = exact_layout(gi, desc->math, desc->algo);
+                R.move_x = L.tc_ok || L.stem_ok || direct_mma_supported(gi, L.dp);
+            } else if (method == GACONV_METHOD_TOP1) {
+                R.move_x = top1_layout(gi).dense || (top1_fused_supported(gi) && gi.c % 4 == 0);
+            } else {
+                R.move_x = topk_of(desc, gi) >= 1 && top1_fused_supported(gi) && gi.c % 4 == 0;
+            }
+            if (R.move_x) R.inner = cl;
+        }
+    }
+    if (R.move_x || R.move_dy) {
+        Geom gi;
+        bool ok = false;
+        if (make_geom(&R.inner, &gi) == GACONV_OK) R.inner_bytes = native_ws_bytes(&R.inner, gi, method, &ok);
+        if (!ok) { R.move_x = R.move_dy = false; R.inner = *desc; R.inner_bytes = 0; }
+    }
+    return R;
+}
+
+// Transposes what has to move into the workspace tail and hands back the inner descriptor and operand pointers.
+// *moved == false: nothing to do, the caller goes on with its own descriptor.
+gaconv_status_t relayout_operands(const void* x, const void* dy, const gaconv_conv_desc_t* desc, int32_t method, cudaStream_t cs,
+                                  gaconv_conv_desc_t* inner, const void** x_out, const void** dy_out, bool* moved)
+{
+    const Relayout R = plan_relayout(desc, method);
+    *moved = R.move_x || R.move_dy;
+    if (!*moved) return GACONV_OK;
     Geom g;
-    st = make_geom(desc, &g);
+    gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
-    void* xt = static_cast<char*>(desc->workspace) + head;
-    if (launch_nchw_to_nhwc(x, xt, g, cs) != cudaSuccess) return GACONV_ERR_CUDA;
-    *inner = *desc;
-    inner->x_layout = GACONV_X_NHWC;
+    const size_t head = align_up(R.inner_bytes, 256);
+    const size_t x_tail = R.move_x ? align_up(x_bytes_of(desc), 256) : 0;
+    st = check_ws(desc, head + x_tail + (R.move_dy ? dy_bytes_of(g) : 0));
+    if (st != GACONV_OK) return st;
+    char* ws = static_cast<char*>(desc->workspace);
+    *x_out = x; *dy_out = dy;
+    if (R.move_x) {
+        if (launch_transpose_batched(x, ws + head, g.c, g.h * g.w, g.n, g.bf16, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        *x_out = ws + head;
+    }
+    if (R.move_dy) {
+        if (launch_transpose_batched(dy, ws + head + x_tail, g.p * g.q, g.k, g.n, g.bf16, cs) != cudaSuccess) return GACONV_ERR_CUDA;
+        *dy_out = ws + head + x_tail;
+    }
+    *inner = R.inner;
     inner->workspace_bytes = head;
-    *x_out = xt;
     return GACONV_OK;
 }
 
@@ -295,9 +335,12 @@ gaconv_status_t gaconv_workspace_size(const gaconv_conv_desc_t* desc, int32_t me
     Geom g;
     gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
-    if (const size_t inner = nchw_relayout_inner_bytes(desc, method)) {      // the channels-last call's scratch, then the transposed X
-        *bytes = align_up(inner, 256) + x_bytes_of(desc);
-        return GACONV_OK;
+    {   // operands that are transposed first: the inner call's scratch, then the transposed copies
+        const Relayout R = plan_relayout(desc, method);
+        if (R.move_x || R.move_dy) {
+            *bytes = align_up(R.inner_bytes, 256) + (R.move_x ? align_up(x_bytes_of(desc), 256) : 0) + (R.move_dy ? dy_bytes_of(g) : 0);
+            return GACONV_OK;
+        }
     }
     switch (method) {
         case GACONV_METHOD_EXACT: *bytes = exact_layout(g, desc->math, desc->algo).total; return GACONV_OK;
@@ -333,10 +376,11 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
     {
         gaconv_conv_desc_t inner;
-        const void* xt = nullptr;
-        st = nchw_relayout(x, desc, GACONV_METHOD_EXACT, static_cast<cudaStream_t>(stream), &inner, &xt);
+        const void *xt = nullptr, *dyt = nullptr;
+        bool moved = false;
+        st = relayout_operands(x, dy, desc, GACONV_METHOD_EXACT, static_cast<cudaStream_t>(stream), &inner, &xt, &dyt, &moved);
         if (st != GACONV_OK) return st;
-        if (xt != nullptr) return gaconv_dw_exact(xt, dy, dw, &inner, stream);
+        if (moved) return gaconv_dw_exact(xt, dyt, dw, &inner, stream);
     }
     const ExactLayout L = exact_layout(g, desc->math, desc->algo);
     const bool mma_ok = direct_mma_supported(g, L.dp);
@@ -385,10 +429,11 @@ gaconv_status_t gaconv_dw_approx(int32_t method, const void* x, const void* dy, 
     if (!aligned16(x) || !aligned16(dy)) return GACONV_ERR_MISALIGNED;
     {
         gaconv_conv_desc_t inner;
-        const void* xt = nullptr;
-        st = nchw_relayout(x, desc, method, cs, &inner, &xt);
+        const void *xt = nullptr, *dyt = nullptr;
+        bool moved = false;
+        st = relayout_operands(x, dy, desc, method, cs, &inner, &xt, &dyt, &moved);
         if (st != GACONV_OK) return st;
-        if (xt != nullptr) return gaconv_dw_approx(method, xt, dy, dw, &inner, seed, stream);
+        if (moved) return gaconv_dw_approx(method, xt, dyt, dw, &inner, seed, stream);
     }
     if (method == GACONV_METHOD_TOPK) {
         // selection of the topk largest magnitudes per map, then the patch accumulation over the retained entries
@@ -442,6 +487,7 @@ gaconv_status_t gaconv_approx_select(const void* dy, int32_t* idx, float* sum, v
     gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
     if (dy == nullptr || idx == nullptr || sum == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (desc->dy_layout == GACONV_DY_NPQK && g.k > 1) return GACONV_ERR_UNSUPPORTED;      // selection alone has no scratch to transpose into
     if (!aligned16(dy) || !aligned16(idx) || !aligned16(sum) || !aligned16(dy_sparse)) return GACONV_ERR_MISALIGNED;
     return launch_select(dy, idx, sum, dy_sparse, g, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GACONV_OK
                                                                                                          : GACONV_ERR_CUDA;
@@ -453,6 +499,7 @@ gaconv_status_t gaconv_approx_select_topk(const void* dy, int32_t* idx, float* s
     gaconv_status_t st = make_geom(desc, &g);
     if (st != GACONV_OK) return st;
     if (dy == nullptr || idx == nullptr || sum == nullptr) return GACONV_ERR_NULL_POINTER;
+    if (desc->dy_layout == GACONV_DY_NPQK && g.k > 1) return GACONV_ERR_UNSUPPORTED;
     if (!aligned16(dy) || !aligned16(idx) || !aligned16(sum)) return GACONV_ERR_MISALIGNED;
     const int t = topk_of(desc, g);
     if (t < 1) return GACONV_ERR_BAD_DESC;

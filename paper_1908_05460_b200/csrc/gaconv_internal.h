@@ -65,8 +65,8 @@ struct Geom {
     int sm_budget;                      // 0: plan for the whole GPU; n > 0: for about n SMs
 };
 
-// ---- N x C x H x W activations -> N x H x W x C (one pass through shared memory) ----
-cudaError_t launch_nchw_to_nhwc(const void* x, void* out, const Geom& g, cudaStream_t stream);
+// ---- out[b][j][i] = in[b][i][j], i < rows, j < cols: N x C x H x W activations -> N x H x W x C, N x P x Q x K gradients -> N x K x P x Q ----
+cudaError_t launch_transpose_batched(const void* in, void* out, int rows, int cols, int batch, bool bf16, cudaStream_t stream);
 
 // ---- fixed-order sum of split partials: dw = alpha * sum_sp partial[sp][0..count) ----
 cudaError_t reduce_splits(const float* partial, float* dw, size_t count, int splits, float alpha, cudaStream_t stream);

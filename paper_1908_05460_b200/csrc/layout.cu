@@ -1,16 +1,17 @@
-// Activations given as N x C x H x W are brought into the N x H x W x C order the tensor-core, stem and gather
-// kernels are built for, by one pass through shared memory into the caller's workspace.  (The paper's own kernel
-// expects channels-last activations as well and pays the same transposition, Sections 2.4 and 3.1.)
+// Operands given in the other order are brought into the kernels' own by one pass through shared memory into the
+// caller's workspace: activations N x C x H x W -> N x H x W x C (what the tensor-core, stem and gather kernels are
+// built for), output gradients N x P x Q x K -> N x K x P x Q.  (The paper's own kernel expects channels-last
+// activations as well and pays the same transposition, Sections 2.4 and 3.1.)
 #include "gaconv_internal.h"
 
 namespace gaconv {
 namespace {
 
-// out[n][j][c] = in[n][c][j], j = h*W + w.  A block turns a 32 x 32 (channel x pixel) tile; both the reads (along
-// the pixels) and the writes (along the channels) are contiguous.
+// out[b][j][i] = in[b][i][j] for i < c, j < hw.  A block turns a 32 x 32 tile; both the reads (along j) and the
+// writes (along i) are contiguous.
 template <typename T>
 __global__ void __launch_bounds__(256)
-nchw_to_nhwc_kernel(const T* __restrict__ in, T* __restrict__ out, int c, int hw)
+transpose_batched_kernel(const T* __restrict__ in, T* __restrict__ out, int c, int hw)
 {
     __shared__ T tile[32][33];
     pdl_release_next_grid();
@@ -28,17 +29,16 @@ nchw_to_nhwc_kernel(const T* __restrict__ in, T* __restrict__ out, int c, int hw
 
 }  // namespace
 
-cudaError_t launch_nchw_to_nhwc(const void* x, void* out, const Geom& g, cudaStream_t stream)
+cudaError_t launch_transpose_batched(const void* in, void* out, int rows, int cols, int batch, bool bf16, cudaStream_t stream)
 {
-    const int hw = g.h * g.w;
-    const dim3 grid((unsigned)((hw + 31) / 32), (unsigned)((g.c + 31) / 32), (unsigned)g.n);
+    const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32), (unsigned)batch);
     if (grid.y > 65535u || grid.z > 65535u) return cudaErrorInvalidValue;
     note_launch();
-    if (g.bf16)
-        return launch_kernel(nchw_to_nhwc_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, dim3(1, 1, 1),
-                             static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(out), g.c, hw);
-    return launch_kernel(nchw_to_nhwc_kernel<float>, grid, dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float*>(x),
-                         static_cast<float*>(out), g.c, hw);
+    if (bf16)
+        return launch_kernel(transpose_batched_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, dim3(1, 1, 1),
+                             static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out), rows, cols);
+    return launch_kernel(transpose_batched_kernel<float>, grid, dim3(256), 0, stream, dim3(1, 1, 1), static_cast<const float*>(in),
+                         static_cast<float*>(out), rows, cols);
 }
 
 }  // namespace gaconv

@@ -142,6 +142,26 @@ def test_nchw_activations_take_the_fast_kernels_through_one_transposing_pass(li,
     assert norm_err(inplace.exact(), ref, dn) <= tol(dtype)
 
 
+# ---- N x P x Q x K output gradients (channels last): transposed once into the workspace, every method ----
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("li", [0, 1, 3, 4], ids=lambda i: NCHW_SHAPES[i].name.replace("nchw", "npqk"))
+@pytest.mark.parametrize("x_layout", [B.X_NHWC, B.X_NCHW], ids=["x-nhwc", "x-nchw"])
+def test_channels_last_output_gradients(li, dtype, x_layout):
+    layer = NCHW_SHAPES[li]
+    x, dy = _inputs(layer, dtype, 145 + li)
+    g = GpuLayer(layer, dtype, x, dy, x_layout=x_layout, dy_layout=B.DY_NPQK, alpha=0.5, topk=2)
+    plain = GpuLayer(layer, dtype, x, dy, alpha=0.5, topk=2)
+    np.testing.assert_array_equal(g.exact(), plain.exact())           # the same kernels on the same values
+    np.testing.assert_array_equal(g.approx(B.METHOD_TOP1), plain.approx(B.METHOD_TOP1))
+    np.testing.assert_array_equal(g.approx(B.METHOD_TOPK), plain.approx(B.METHOD_TOPK))
+    ref, dn = oracle.dw_exact(to_f64(x), to_f64(dy), oshape(layer), 0.5)
+    assert norm_err(g.exact(), ref, dn) <= tol(dtype)
+    with pytest.raises(B.GaconvError) as e:                            # the selection-only entry has no scratch to transpose into
+        g.select()
+    assert e.value.status == B.ERR_UNSUPPORTED
+    assert B.gaconv_poll_async_status(g.desc) == B.OK
+
+
 def test_selection_ties_and_planted_maxima():
     layer = ConvLayer("ties", 4, 2, 32, 32, 8, 3, 3, 1, 1)
     for dtype in DTYPES:
