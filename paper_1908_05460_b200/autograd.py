@@ -51,13 +51,13 @@ class GAConv2d(torch.nn.Module):
     def forward(self, x):
         return _Conv2dFilterGrad.apply(x.contiguous(memory_format=torch.channels_last), self.weight, self)
 
-    def _desc(self, x):
-        key = (tuple(x.shape), x.dtype)
+    def _desc(self, x, dy_layout=B.DY_NKPQ):
+        key = (tuple(x.shape), x.dtype, dy_layout)
         if key not in self._desc_cache:
             n, c, h, w = x.shape
             k = self.weight.shape[0]
             layer = ConvLayer("gaconv2d", n, c, h, w, k, self.kernel_size, self.kernel_size, self.stride, self.padding)
-            d = B.make_desc(layer, x.dtype, x_layout=B.X_NHWC, dw_layout=B.DW_KCRS, alpha=1.0)
+            d = B.make_desc(layer, x.dtype, x_layout=B.X_NHWC, dw_layout=B.DW_KCRS, alpha=1.0, dy_layout=dy_layout)
             self._desc_cache[key] = (d, B.attach_workspace(d, methods=(B.METHOD_EXACT, B.METHOD_TOP1), device=x.device))
         return self._desc_cache[key][0]
 
@@ -65,11 +65,15 @@ class GAConv2d(torch.nn.Module):
         """dW [K,C,R,S] (the weight's dtype) of this layer for activations x and output gradient dy."""
         B.load()
         x = x.contiguous(memory_format=torch.channels_last)        # NHWC memory under an NCHW-shaped tensor
-        dy = dy.contiguous()                                       # [N,K,P,Q]
         if dy.dtype != x.dtype:
             dy = dy.to(x.dtype)
+        # the gradient of a channels-last forward arrives channels-last: the library takes it as it is ([N,P,Q,K] memory)
+        if dy.dim() == 4 and dy.shape[1] > 1 and not dy.is_contiguous() and dy.is_contiguous(memory_format=torch.channels_last):
+            dy_layout = B.DY_NPQK
+        else:
+            dy, dy_layout = dy.contiguous(), B.DY_NKPQ             # [N,K,P,Q]
         dw = torch.empty(self.weight.shape, dtype=torch.float32, device=x.device)
-        d = self._desc(x)
+        d = self._desc(x, dy_layout)
         if self.schedule is None:
             B.gaconv_dw_exact(x, dy, dw, d)
         else:
