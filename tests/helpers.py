@@ -28,7 +28,7 @@ class GpuLayer:
 
     def __init__(self, layer: ConvLayer, dtype, x_nchw: torch.Tensor, dy: torch.Tensor, *, x_layout=B.X_NHWC,
                  dw_layout=B.DW_KRSC, alpha=1.0, rand_std=1.0 / 128, algo=B.ALGO_AUTO, math=B.MATH_DEFAULT, topk=1,
-                 dy_layout=B.DY_NKPQ):
+                 dy_layout=B.DY_NKPQ, sm_budget=0):
         self.layer, self.dtype, self.dw_layout = layer, dtype, dw_layout
         self.x = (I.to_nhwc(x_nchw) if x_layout == B.X_NHWC else x_nchw.contiguous()).cuda()
         self.dy = (dy.contiguous() if dy_layout == B.DY_NKPQ else dy.permute(0, 2, 3, 1).contiguous()).cuda()
@@ -36,7 +36,7 @@ class GpuLayer:
                  B.DW_RSCK: (layer.r, layer.s, layer.c, layer.k)}[dw_layout]
         self.dw = torch.full(shape, float("nan"), dtype=torch.float32, device="cuda")
         self.desc = B.make_desc(layer, dtype, x_layout=x_layout, dw_layout=dw_layout, alpha=alpha, rand_std=rand_std,
-                                algo=algo, math=math, topk=topk, dy_layout=dy_layout)
+                                algo=algo, math=math, topk=topk, dy_layout=dy_layout, sm_budget=sm_budget)
         self.ws = B.attach_workspace(self.desc)
 
     def logical_dw(self) -> np.ndarray:

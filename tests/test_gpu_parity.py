@@ -334,6 +334,19 @@ def test_full_size_layers(net, li, batch, dtype):
         worst = max(worst, abs(got[k, c, r, s_] - v) / nrm)
     assert worst <= tol(dtype)
     assert np.all(np.isfinite(got))
+    # the same layer as the benchmark's step launches it: sized for its share of the SMs (148 * roofline time / 12,
+    # between 18 and 74), which changes the splits, the clusters and the top-1 grid
+    eb = 2 if dtype == torch.bfloat16 else 4
+    t_roof = max(layer.flops_exact() / (1654.6e12 * (1.0 if eb == 2 else 0.5)), layer.bytes_exact(eb) / 6456.2e9) * 1e6
+    gb = GpuLayer(layer, dtype, x, dy, sm_budget=max(18, min(74, int(148 * t_roof / 12.0))))
+    assert norm_err(gb.approx(B.METHOD_TOP1), ref, dn) <= top1_bound(layer, dtype)
+    got = gb.exact()
+    worst = 0.0
+    for (k, c, r, s_) in picks:
+        v, nrm = oracle.dw_exact_at(xd, dyd, sh, k, c, r, s_)
+        worst = max(worst, abs(got[k, c, r, s_] - v) / nrm)
+    assert worst <= tol(dtype)
+    assert np.all(np.isfinite(got)) and B.gaconv_poll_async_status(gb.desc) == B.OK
 
 
 # ---- tensor-core (tcgen05) exact path, forced, on shapes that exercise each of its tilings ----
