@@ -244,7 +244,7 @@ Relayout plan_relayout(const gaconv_conv_desc_t* desc, int32_t method)
     R.inner = *desc;
     const bool reads_inputs = method == GACONV_METHOD_EXACT || method == GACONV_METHOD_TOP1 || method == GACONV_METHOD_TOPK;
     if (!reads_inputs) return R;
-    R.move_dy = desc->dy_layout == GACONV_DY_NPQK && desc->k > 1 && (long long)desc->h * desc->w > 0;
+    R.move_dy = desc->dy_layout == GACONV_DY_NPQK && desc->k > 1;          // (one output channel: the two orders coincide)
     R.inner.dy_layout = GACONV_DY_NKPQ;
     if (desc->x_layout == GACONV_X_NCHW && desc->c >= 2 && desc->algo != GACONV_ALGO_DIRECT) {
         gaconv_conv_desc_t cl = R.inner;

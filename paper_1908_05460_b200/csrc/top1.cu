@@ -5,8 +5,11 @@
 //                     equals) and the signed sum of the map      [Algorithm 1, arg-max and sum lines]
 //   gather_kernel  -- dW[k,r,s,c] = alpha * sum_n sum[n,k] * Xz[n, c, patch at the selected position]
 //                                                                  [Algorithm 1, accumulation line]
+// The top-k variant (Section 2.3, last sentence) selects with select_topk_kernel and feeds the list to
+// top1_fused_kernel (k records per image), or to gather_kernel when the records do not fit shared memory;
+// select_sparse_transposed_kernel writes the sparse tensor the dense route contracts on small maps.
 // Selection compares the bit pattern of |v| in the input dtype as an unsigned integer, which orders
-// finite values exactly as their magnitudes do, so indices are reproducible bit for bit.
+// finite values exactly as their magnitudes do (NaN above Inf), so indices are reproducible bit for bit.
 #include <cooperative_groups.h>
 
 #include "gaconv_internal.h"
