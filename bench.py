@@ -590,8 +590,14 @@ def main():
         t = sum_us["top1"]
         fams["top1"] = {"bound": "hbm", "achieved": sum(r["top1_bytes"] for r in table) / t / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": sum(r["top1_bytes"] for r in table) / (peaks["hbm_gbs"] * 1e3) / t, "layers": len(table), "sum_us": t}
-        dom = max(fams, key=lambda f: fams[f]["sum_us"])
-        kernel = {"exact_tensor_bound": "exact_tc_kernel", "exact_hbm_bound": "exact_tc_kernel", "top1": "top1_fused_kernel"}[dom]
+        # the dominant kernel first (the exact families are both mostly exact_tc_kernel launches, as in the ncu launch
+        # list of the step), then that kernel's larger family
+        kernel_of = {"exact_tensor_bound": "exact_tc_kernel", "exact_hbm_bound": "exact_tc_kernel", "top1": "top1_fused_kernel"}
+        per_kernel = {}
+        for f, v in fams.items():
+            per_kernel[kernel_of[f]] = per_kernel.get(kernel_of[f], 0.0) + v["sum_us"]
+        kernel = max(per_kernel, key=per_kernel.get)
+        dom = max((f for f in fams if kernel_of[f] == kernel), key=lambda f: fams[f]["sum_us"])
         roof = {k: fams[dom][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
         roof.update({"kernel": kernel, "family": dom, "peak_source": peaks["source"], "families": fams,
                      "traffic": traffic_from_profiles(kernel, dom)})
