@@ -785,8 +785,14 @@ bool choose_splits(TcParams& P, const Geom& g, int tiles)
     for (int c = 1; c <= 4; ++c)
         if (sp_of[c] > 0 && (fits[c] || !any_fit)) most = std::max(most, sp_of[c]);
     int cl = 0, splits = 0;
+    // (the shortcut only while a CTA's share of the reduction is short -- up to ~160 k-steps, 128->... at batch 128;
+    //  with more work per CTA the idle SMs cost more than the workspace pass: 256->256@8x8 at batch 256, 26 us against 30)
+    const long long total_ksteps = (long long)P.chunks * P.ksteps;
     for (int c = 4; c >= 1 && cl == 0; --c)
-        if ((fits[c] || !any_fit) && per_of[c] == 1 && sp_of[c] * 10 >= most * 6) { cl = c; splits = sp_of[c]; }
+        if ((fits[c] || !any_fit) && per_of[c] == 1 && sp_of[c] * 10 >= most * 6 &&
+            (sp_of[c] == most || g.sm_budget > 0 || total_ksteps <= 160LL * sp_of[c])) {      // (with a budget the other SMs are not idle)
+            cl = c; splits = sp_of[c];
+        }
     for (int c = 4; c >= 1 && cl == 0; --c)
         if ((fits[c] || !any_fit) && sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
     if (cl == 0) return false;
