@@ -763,7 +763,10 @@ bool choose_splits(TcParams& P, const Geom& g, int tiles)
         if (max_splits < 1) max_splits = 1;
     }
     if (max_splits > P.chunks) max_splits = P.chunks;
-    const int cl_cap = env_int("GACONV_TC_CLUSTER", 4);
+    // Sharing the GPU (a budget): no clusters.  The launch is then main-loop-bound on its few SMs, and the cluster
+    // barriers and the pull through distributed shared memory cost it more than the workspace pass of the second
+    // kernel (measured on the 58-layer step: exact phase 540 -> 526 us).
+    const int cl_cap = g.sm_budget > 0 ? 1 : env_int("GACONV_TC_CLUSTER", 4);
     // Measured on the layer shapes of the three networks: a cluster whose splits cover the whole tile (no workspace,
     // no second kernel) wins even at two thirds of the CTAs; otherwise the largest cluster that keeps 85% of them.
     const int cl_force = env_int("GACONV_TC_FORCE_CL", 0);
