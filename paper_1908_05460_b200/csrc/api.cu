@@ -103,14 +103,15 @@ private:
     std::vector<std::pair<PlanKey, L>> e_;
 };
 
-// Maps of at most 4x4 pixels with many channels: the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes,
+// Small maps with many channels (up to 4x4 pixels from 128 channels, up to 8x8 from 256): the N*K patch accumulations (N*K*R*S*C FMAs on the FP32 pipes,
 // the same number of bytes gathered from L2) cost more than the dense contraction on tensor cores, and with so few
 // pixels per map the sparse tensor is not that sparse (1 - 1/(PQ), Section 2.3).  Then the method is run
 // literally as the paper states it: build the sparse version of dY (one entry per map, the signed sum) and take
-// its exact filter gradient with the tensor-core kernel.  (On 8x8 maps the gather kernel measured faster.)
+// its exact filter gradient with the tensor-core kernel.  (8x8 maps: the gather kernel is faster with 128 channels;
+// with 256 the two tie alone and the dense route is cheaper among other layers, so it is taken from 256 channels on.)
 bool top1_dense_route(const Geom& g, TcPlan* tp)
 {
-    return g.bf16 && g.p * g.q <= 16 && g.c >= 128 && plan_tc(g, tp);
+    return g.bf16 && ((g.p * g.q <= 16 && g.c >= 128) || (g.p * g.q <= 64 && g.c >= 256)) && plan_tc(g, tp);
 }
 
 struct Top1Layout { size_t idx_off, sum_off, partial_off, sparse_off, scratch_off, total; GatherPlan gp; TcPlan tp; bool dense; };

@@ -28,7 +28,8 @@ def top1_bound(layer, dtype):
     at least 128 input channels take the route 'sparse dY + dense tensor-core kernel', which rounds each sum to
     bf16 once (8 significant bits, round to nearest: at most 2^-8 |sum| <= 2^-8 sum|dY| per image, i.e. 2^-8 of the
     normaliser), plus the fp32 terms."""
-    dense = dtype == torch.bfloat16 and layer.p * layer.q <= 16 and layer.c >= 128
+    pq = layer.p * layer.q
+    dense = dtype == torch.bfloat16 and ((pq <= 16 and layer.c >= 128) or (pq <= 64 and layer.c >= 256))
     return 2.0 ** -8 + 1e-4 if dense else 1e-5
 
 
