@@ -220,7 +220,7 @@ bool make_params(const Geom& g, StemParams* out)
     P.win_h = (bp - 1) * g.stride_h + g.r;
     if (P.box_w > 256 || P.win_h > 256) return false;
     P.nt = (ncols + 7) / 8;
-    int splits = (148 * 4) / P.tiles_k;
+    int splits = (148 * (ncols <= 32 ? 8 : 4)) / P.tiles_k;     // (3x3 stems: eight light CTAs per SM hide the fragment latency better)
     if (splits < 1) splits = 1;
     if (splits > P.items) splits = P.items;
     const int per = (P.items + splits - 1) / splits;
