@@ -796,6 +796,10 @@ bool choose_splits(TcParams& P, const Geom& g, int tiles)
             (sp_of[c] == most || g.sm_budget > 0 || total_ksteps <= 160LL * sp_of[c])) {      // (with a budget the other SMs are not idle)
             cl = c; splits = sp_of[c];
         }
+    // The tile needs the second kernel anyway.  With a long main loop per CTA (60 k-steps and more) no clusters at
+    // all measured faster -- every SM gets a CTA and nobody waits at a cluster barrier (128->128@16x16 20.8 -> 19.6 us,
+    // 64->64@32x32 26.4 -> 24.5, 5x5 64->64@16x16 18.7 -> 16.8); with short loops the larger workspace pass loses.
+    if (cl == 0 && sp_of[1] == most && (fits[1] || !any_fit) && total_ksteps >= 60LL * most) { cl = 1; splits = sp_of[1]; }
     for (int c = 4; c >= 1 && cl == 0; --c)
         if ((fits[c] || !any_fit) && sp_of[c] > 0 && sp_of[c] * 100 >= most * 85) { cl = c; splits = sp_of[c]; }
     if (cl == 0) return false;
