@@ -375,6 +375,31 @@ gaconv_status_t gaconv_dw_exact(const void* x, const void* dy, float* dw, const 
     if (x == nullptr || dy == nullptr || dw == nullptr) return GACONV_ERR_NULL_POINTER;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(dw)) return GACONV_ERR_MISALIGNED;
     if (desc->math == GACONV_MATH_TF32 && g.bf16) return GACONV_ERR_BAD_DESC;
+    if (desc->dy_layout == GACONV_DY_NPQK && g.k > 1 && desc->algo != GACONV_ALGO_DIRECT) {
+        // Small maps: the tensor-core kernel's dY operand IS the channels-last order (its pre-pass would transpose an
+        // N x K x P x Q gradient into it), so a channels-last gradient is read where it lies; only X may have to move.
+        const Relayout R = plan_relayout(desc, GACONV_METHOD_EXACT);
+        Geom gi;
+        if (make_geom(&R.inner, &gi) == GACONV_OK) {
+            const ExactLayout Li = exact_layout(gi, desc->math, desc->algo);
+            if (Li.tc_ok && Li.tp.reads_transposed_dy) {
+                const size_t head = align_up(Li.total, 256);
+                st = check_ws(desc, head + (R.move_x ? x_bytes_of(desc) : 0));
+                if (st != GACONV_OK) return st;
+                char* ws = static_cast<char*>(desc->workspace);
+                const void* xs = x;
+                if (R.move_x) {
+                    if (launch_transpose_batched(x, ws + head, g.c, g.h * g.w, g.n, g.bf16, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+                        return GACONV_ERR_CUDA;
+                    xs = ws + head;
+                }
+                cudaError_t e = launch_tc(xs, nullptr, dw, reinterpret_cast<float*>(ws + Li.partial_off), const_cast<void*>(dy),
+                                          reinterpret_cast<uint32_t*>(ws + kWsCounterOffset), reinterpret_cast<uint32_t*>(ws), Li.tp,
+                                          static_cast<cudaStream_t>(stream));
+                return e == cudaSuccess ? GACONV_OK : GACONV_ERR_CUDA;
+            }
+        }
+    }
     {
         gaconv_conv_desc_t inner;
         const void *xt = nullptr, *dyt = nullptr;
